@@ -1,0 +1,134 @@
+/*
+ * ptq.h -- C ABI of the B200 (sm_100a) per-layer quantizer: sensitivity-ordered, row-parallel
+ * quantization with one shared inverse Hessian (Sec. 4 of the paper).
+ *
+ * Data model (Sec. 3): W is [rows x cols] = d_row x d_col, X is [cols x n] = d_col x N, the layer
+ * computes W X and the objective is ||W X - What X||^2 (Eq. 2).
+ *
+ * Rules common to every entry point
+ *   - Every data pointer is a DEVICE pointer owned by the caller (unless a parameter says "host").
+ *     The library allocates no device memory: scratch comes from the caller's workspace `ws`, whose
+ *     minimum size is given by ptq_workspace_bytes().  Base pointers must be 16-byte aligned.
+ *   - Matrices are row-major.  H, Hinv: float64 [cols x cols], full symmetric storage.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*).  The return value reports
+ *     argument errors found on the host (nothing is launched then).  Conditions found on the device
+ *     (not positive definite, non-finite input, bounded wait expired) are recorded in the caller's
+ *     `status` word, int32[4] = {code, index, aux, 0}; the first error sticks, so the caller zeroes it
+ *     before a sequence of calls and reads it after synchronising the stream.
+ *   - Inputs are never modified; outputs are fully overwritten (H of ptq_hessian_accumulate is updated).
+ *   - Results are deterministic: fixed reduction orders, no floating-point atomics.
+ *   - No exceptions, no exit(), no stdout, no device trap, no unbounded device-side wait.
+ */
+#ifndef PTQ_H_
+#define PTQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    PTQ_OK = 0,
+    PTQ_ERR_INVALID_ARG = 1,
+    PTQ_ERR_ALIGNMENT = 2,
+    PTQ_ERR_WORKSPACE = 3,
+    PTQ_ERR_NOT_SPD = 4,     /* status[1] = failing pivot index */
+    PTQ_ERR_NONFINITE = 5,
+    PTQ_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired */
+    PTQ_ERR_CUDA = 7,        /* a CUDA runtime call failed on the host */
+    PTQ_ERR_UNSUPPORTED = 8
+} ptq_status;
+
+/* Damping (Implementation Details: a constant is added to the diagonal of H). */
+typedef enum {
+    PTQ_DAMP_REL_MEAN_DIAG = 0, /* lambda = damp * mean(diag H) */
+    PTQ_DAMP_ABS = 1            /* lambda = damp (the paper's 0.1) */
+} ptq_damp_mode;
+
+/* Column score (Sec. 4.1 names the keys err / w / sensi; Sec. 4.2 step 2 sums them per column). */
+typedef enum {
+    PTQ_SCORE_QERR = 0,  /* Eq. 10: (w - quant(w))^2 / (2 [Hinv]_jj)   (default) */
+    PTQ_SCORE_PRUNE = 1, /* Eq. 8 :  w^2 / (2 [Hinv]_jj) */
+    PTQ_SCORE_ERR = 2,   /* (w - quant(w))^2 */
+    PTQ_SCORE_W = 3,     /* w^2 */
+    PTQ_SCORE_NONE = 4   /* no sorting: identity order */
+} ptq_score_mode;
+
+typedef enum {
+    PTQ_CALL_HESSIAN_ACCUMULATE = 0,
+    PTQ_CALL_PREPARE_HINV = 1,
+    PTQ_CALL_SENSITIVITY_ORDER = 2,
+    PTQ_CALL_QUANTIZE_LAYER = 3,
+    PTQ_CALL_HESSIAN_ACCUMULATE_F64 = 4
+} ptq_call_id;
+
+/* Minimum workspace, in bytes, for one call with these sizes (host function, no CUDA calls). */
+size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n);
+
+/*
+ * H += 2 * X X^T  (Sec. 3: the second derivative of Eq. 2 with respect to one row of W).
+ *   H    [cols x cols] float64, in/out; the caller zeroes it before the first chunk of calibration columns
+ *   X    [cols x n]    float32, row stride ldx >= n elements (vector loads are used when X is 16-byte aligned
+ *                      and ldx is a multiple of 4)
+ * The product is formed on the tensor cores from error-free integer slices of X, so H carries
+ * float64-level accuracy (relative error about 1e-12 or better).
+ */
+int ptq_hessian_accumulate(double *H, const float *X, int cols, int n, int64_t ldx, void *ws, size_t ws_bytes,
+                           int32_t *status, void *stream);
+
+/* Same contract, computed with float64 FMAs (cross-check of the tensor-core path). */
+int ptq_hessian_accumulate_f64(double *H, const float *X, int cols, int n, int64_t ldx, void *ws, size_t ws_bytes,
+                               int32_t *status, void *stream);
+
+/*
+ * Hinv = (H + lambda I)^-1 by Cholesky factorisation and inversion of the factor (Sec. 5 item 1).
+ *   H          [cols x cols] float64, const
+ *   Hinv       [cols x cols] float64, out
+ *   Hinv_diag  [cols] float64, out (the diagonal of Hinv, what the sensitivities need)
+ *   lambda_out [1] float64, out (device)
+ * A non-positive pivot sets status = {PTQ_ERR_NOT_SPD, pivot index}.
+ */
+int ptq_prepare_hinv(const double *H, int cols, int damp_mode, double damp, double *Hinv, double *Hinv_diag,
+                     double *lambda_out, void *ws, size_t ws_bytes, int32_t *status, void *stream);
+
+/*
+ * Helper: per-row asymmetric min-max grid whose range always contains 0, from the original W
+ * (Sec. 3, OBQ paragraph: a fixed grid of width Delta).  scale, zero: [rows] float32, out.
+ * quant_i(w) = scale_i * (clamp(rint(w / scale_i) + zero_i, 0, 2^bits - 1) - zero_i), rint = ties to even.
+ */
+int ptq_minmax_grid(const float *W, int rows, int cols, int64_t ldw, int bits, float *scale, float *zero,
+                    int32_t *status, void *stream);
+
+/*
+ * Sec. 4.2 steps 1-3: S_j = sum_i score(w_ij) from the original W and diag(Hinv); perm = columns by S descending,
+ * equal scores keep the lower column index first.   S [cols] float64 out, perm [cols] int32 out.
+ */
+int ptq_sensitivity_order(const float *W, int rows, int cols, int64_t ldw, const double *Hinv_diag, const float *scale,
+                          const float *zero, int bits, int score_mode, double *S, int32_t *perm, void *ws,
+                          size_t ws_bytes, int32_t *status, void *stream);
+
+/*
+ * Sec. 4.2 steps 3-5: permute W and Hinv by perm, then quantize one column at a time, all rows in parallel;
+ * after each column the remaining columns absorb the error (Eq. 11) and the shared inverse Hessian is
+ * updated (Eq. 12).  The updates are applied in blocked form through the upper Cholesky factor of the
+ * permuted inverse Hessian, whose row p equals row p of the Eq.-12-updated matrix divided by the square
+ * root of its pivot.
+ *   codes      [rows x cols] uint8, out, one code per byte, ORIGINAL column order
+ *   What       [rows x cols] float32, out (may be NULL): scale_i * (code - zero_i)
+ *   H_undamped [cols x cols] float64 and loss_out [1] float64 (device): loss = ||W X - What X||^2
+ *              = 1/2 tr(dW H dW^T); pass NULL for either to skip
+ */
+int ptq_quantize_layer(const float *W, int rows, int cols, int64_t ldw, const double *Hinv, const int32_t *perm,
+                       const float *scale, const float *zero, int bits, uint8_t *codes, float *What,
+                       const double *H_undamped, double *loss_out, void *ws, size_t ws_bytes, int32_t *status,
+                       void *stream);
+
+const char *ptq_status_string(int code);
+int ptq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PTQ_H_ */

@@ -1,0 +1,237 @@
+// C-ABI entry points (see include/ptq.h): argument checks, workspace carving, kernel sequencing.
+#include "common.cuh"
+#include "dgemm.cuh"
+#include "chol.cuh"
+#include "order.cuh"
+#include "colloop.cuh"
+#include "gram.cuh"
+
+using namespace ptq;
+
+namespace {
+
+__global__ void convert_f32_f64_kernel(const float* __restrict__ X, int rows, int n, int64_t ldx,
+                                       double* __restrict__ Xd) {
+    const int i = blockIdx.y;
+    for (int k = blockIdx.x * blockDim.x + threadIdx.x; k < n; k += gridDim.x * blockDim.x)
+        Xd[(int64_t)i * n + k] = (double)X[(int64_t)i * ldx + k];
+}
+
+inline int grid_x_for(int n, int threads) {
+    int g = cdiv(n, threads);
+    return g < 1 ? 1 : (g > 1024 ? 1024 : g);
+}
+
+size_t loss_partials_count(int rows, int cols) { return (size_t)cdiv(rows, 64) * cdiv(cols, 64); }
+
+}  // namespace
+
+extern "C" {
+
+int ptq_version(void) { return 1; }
+
+const char* ptq_status_string(int code) {
+    switch (code) {
+        case PTQ_OK: return "ok";
+        case PTQ_ERR_INVALID_ARG: return "invalid argument";
+        case PTQ_ERR_ALIGNMENT: return "pointer or leading dimension not aligned";
+        case PTQ_ERR_WORKSPACE: return "workspace too small";
+        case PTQ_ERR_NOT_SPD: return "matrix not positive definite";
+        case PTQ_ERR_NONFINITE: return "non-finite value";
+        case PTQ_ERR_TIMEOUT: return "bounded device wait expired";
+        case PTQ_ERR_CUDA: return "CUDA runtime error";
+        case PTQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        default: return "unknown status";
+    }
+}
+
+size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
+    if (cols < 1) return 0;
+    const size_t c = (size_t)cols;
+    size_t total = 0;
+    auto add = [&](size_t bytes) { total += align_up(bytes); };
+    switch (call_id) {
+        case PTQ_CALL_HESSIAN_ACCUMULATE:
+            if (n < 1) return 0;
+            return gram_workspace_bytes(cols, n);
+        case PTQ_CALL_HESSIAN_ACCUMULATE_F64:
+            if (n < 1) return 0;
+            add(c * (size_t)n * sizeof(double));
+            break;
+        case PTQ_CALL_PREPARE_HINV:
+            add(c * c * sizeof(double));
+            add(c * c * sizeof(double));
+            break;
+        case PTQ_CALL_SENSITIVITY_ORDER:
+            if (rows < 1) return 0;
+            add((size_t)cdiv(rows, kScoreRowChunk) * c * sizeof(double));
+            break;
+        case PTQ_CALL_QUANTIZE_LAYER:
+            if (rows < 1) return 0;
+            add(c * c * sizeof(double));                    // permuted inverse Hessian -> its factor U
+            add((size_t)rows * c * sizeof(double));         // permuted W (float64), later dW
+            add((size_t)rows * c * sizeof(double));         // scaled errors E
+            add((size_t)rows * c);                          // codes in permuted order
+            add(c * sizeof(int32_t));                       // flags
+            add(c * sizeof(int32_t));                       // inverse permutation
+            add(loss_partials_count(rows, cols) * sizeof(double));
+            break;
+        default:
+            return 0;
+    }
+    return total;
+}
+
+int ptq_hessian_accumulate_f64(double* H, const float* X, int cols, int n, int64_t ldx, void* ws, size_t ws_bytes,
+                               int32_t* status, void* stream_) {
+    (void)status;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!H || !X || cols < 1 || n < 1 || ldx < n) return PTQ_ERR_INVALID_ARG;
+    if (!aligned16(H) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE_F64, 0, cols, n)) return PTQ_ERR_WORKSPACE;
+    Carver cv(ws);
+    double* Xd = cv.take<double>((size_t)cols * n);
+    convert_f32_f64_kernel<<<dim3(grid_x_for(n, 256), cols), 256, 0, stream>>>(X, cols, n, ldx, Xd);
+    GemmParams g = gemm_defaults();
+    g.A = Xd; g.lda = n; g.a_trans = 0;
+    g.B = Xd; g.ldb = n; g.b_trans = 1;
+    g.C = H; g.ldc = cols;
+    g.M = cols; g.N = cols; g.K = n;
+    g.alpha = 2.0; g.beta = 1.0; g.upper_only = 1; g.mirror = 1;
+    return launch_dgemm(g, 1, stream);
+}
+
+int ptq_hessian_accumulate(double* H, const float* X, int cols, int n, int64_t ldx, void* ws, size_t ws_bytes,
+                           int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!H || !X || cols < 1 || n < 1 || ldx < n) return PTQ_ERR_INVALID_ARG;
+    if (!aligned16(H) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE, 0, cols, n)) return PTQ_ERR_WORKSPACE;
+    return gram_accumulate(H, X, cols, n, ldx, ws, status, stream);
+}
+
+int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, double* Hinv, double* Hinv_diag,
+                     double* lambda_out, void* ws, size_t ws_bytes, int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!H || !Hinv || !Hinv_diag || !lambda_out || cols < 1 || !(damp >= 0.0)) return PTQ_ERR_INVALID_ARG;
+    if (damp_mode != PTQ_DAMP_REL_MEAN_DIAG && damp_mode != PTQ_DAMP_ABS) return PTQ_ERR_INVALID_ARG;
+    if (!aligned16(H) || !aligned16(Hinv) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_PREPARE_HINV, 0, cols, 0)) return PTQ_ERR_WORKSPACE;
+    const int n = cols;
+    Carver cv(ws);
+    double* R = cv.take<double>((size_t)n * n);
+    double* V = cv.take<double>((size_t)n * n);
+    lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status);
+    damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out);
+    int st = cholesky_upper(R, n, status, stream);
+    if (st) return st;
+    if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
+    st = trtri_upper(R, V, Hinv, n, stream);
+    if (st) return st;
+    st = lauum_upper(V, Hinv, n, stream);
+    if (st) return st;
+    extract_diag_kernel<<<cdiv(n, 256), 256, 0, stream>>>(Hinv, n, Hinv_diag);
+    return launch_status();
+}
+
+int ptq_minmax_grid(const float* W, int rows, int cols, int64_t ldw, int bits, float* scale, float* zero,
+                    int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!W || !scale || !zero || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8)
+        return PTQ_ERR_INVALID_ARG;
+    minmax_grid_kernel<<<rows, 256, 0, stream>>>(W, rows, cols, ldw, bits, scale, zero, status);
+    return launch_status();
+}
+
+int ptq_sensitivity_order(const float* W, int rows, int cols, int64_t ldw, const double* Hinv_diag, const float* scale,
+                          const float* zero, int bits, int score_mode, double* S, int32_t* perm, void* ws,
+                          size_t ws_bytes, int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!W || !S || !perm || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8) return PTQ_ERR_INVALID_ARG;
+    if (score_mode < PTQ_SCORE_QERR || score_mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
+    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_PRUNE) && !Hinv_diag) return PTQ_ERR_INVALID_ARG;
+    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_ERR) && (!scale || !zero)) return PTQ_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_SENSITIVITY_ORDER, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
+    if (!aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    Carver cv(ws);
+    const int chunks = cdiv(rows, kScoreRowChunk);
+    double* partial = cv.take<double>((size_t)chunks * cols);
+    if (score_mode != PTQ_SCORE_NONE)
+        score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
+                                                                              score_mode, partial);
+    score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status);
+    rank_sort_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(S, cols, perm);
+    return launch_status();
+}
+
+int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const double* Hinv, const int32_t* perm,
+                       const float* scale, const float* zero, int bits, uint8_t* codes, float* What,
+                       const double* H_undamped, double* loss_out, void* ws, size_t ws_bytes, int32_t* status,
+                       void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!W || !Hinv || !perm || !scale || !zero || !codes || rows < 1 || cols < 1 || ldw < cols || bits < 2 ||
+        bits > 8)
+        return PTQ_ERR_INVALID_ARG;
+    if (!aligned16(Hinv) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaFuncSetAttribute(colloop_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kColloopSmem);
+        attr_done = true;
+    }
+    const int n = cols;
+    Carver cv(ws);
+    double* U = cv.take<double>((size_t)n * n);
+    double* Wp = cv.take<double>((size_t)rows * n);
+    double* E = cv.take<double>((size_t)rows * n);
+    uint8_t* codes_p = cv.take<uint8_t>((size_t)rows * n);
+    int32_t* flags = cv.take<int32_t>(n);
+    int32_t* invperm = cv.take<int32_t>(n);
+    double* partials = cv.take<double>(loss_partials_count(rows, cols));
+
+    // flags and invperm are adjacent pieces of the workspace: clear both
+    if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
+        cudaSuccess)
+        return PTQ_ERR_CUDA;
+    perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status);
+    gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U);
+    gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp);
+    int st = cholesky_upper(U, n, status, stream);   // blocked Eq. 12
+    if (st) return st;
+
+    const int row_ctas = cdiv(rows, kRowsPerCta);
+    for (int p0 = 0; p0 < n; p0 += kNB) {
+        const int kb = n - p0 < kNB ? n - p0 : kNB;
+        colloop_block_kernel<<<row_ctas, 128, kColloopSmem, stream>>>(Wp, rows, n, p0, kb, U, scale, zero, bits, E,
+                                                                      codes_p);
+        const int rest = n - p0 - kb;
+        if (rest <= 0) break;
+        GemmParams g = gemm_defaults();     // deferred Eq. 11: W[:, later] -= E[:, block] U[block, later]
+        g.A = E + p0; g.lda = n; g.a_trans = 0;
+        g.B = U + (int64_t)p0 * n + p0 + kb; g.ldb = n; g.b_trans = 0;
+        g.C = Wp + p0 + kb; g.ldc = n;
+        g.M = rows; g.N = rest; g.K = kb;
+        g.alpha = -1.0; g.beta = 1.0;
+        st = launch_dgemm(g, 1, stream);
+        if (st) return st;
+    }
+
+    const bool want_loss = H_undamped && loss_out;
+    double* dW = want_loss ? Wp : nullptr;
+    finalize_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(codes_p, invperm, W, rows, n, ldw, scale, zero,
+                                                                       codes, What, dW);
+    if (want_loss) {
+        GemmParams g = gemm_defaults();     // sum_ij (dW H)_ij dW_ij
+        g.A = dW; g.lda = n; g.a_trans = 0;
+        g.B = H_undamped; g.ldb = n; g.b_trans = 0;
+        g.M = rows; g.N = n; g.K = n;
+        g.D = dW; g.ldd = n; g.partials = partials;
+        dim3 grid;
+        st = launch_dgemm(g, 1, stream, 64, &grid);
+        if (st) return st;
+        sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y), 0.5, loss_out);
+    }
+    return launch_status();
+}
+
+}  // extern "C"

@@ -1,0 +1,468 @@
+// H += 2 X X^T on the 5th-generation tensor cores, to float64 accuracy (Sec. 3: the Hessian of Eq. 2).
+//
+// The column order and the rounding decisions of the method are sensitive to errors in H far below
+// float32 resolution, so the product is formed from error-free integer slices:
+//   every row x_i of X is scaled by a power of two 2^sh_i so that |x| 2^sh_i < 2^46, rounded to an integer v
+//   (exact for float32 data within 2^-46 of the row maximum) and written as six balanced base-256 digits,
+//       v = sum_{s=0..5} d_s 256^(5-s),  d_s in [-128, 127]  (int8 "slices", most significant first).
+//   Then  sum_k v_ik v_jk = sum_{a,b} 256^(10-a-b) (D_a D_b^T)_ij, and each D_a D_b^T is an exact int8 x int8 -> int32
+//   tensor-core product.  Slice pairs with a + b = t share the weight 256^(10-t), so one int32 accumulator G_t per
+//   group t is enough; groups t <= 5 are kept (21 pair products), the dropped ones weigh 2^-48 and less.
+//
+// Kernel: one 128 x 64 output tile per CTA iteration (upper triangle only, mirrored on store).  A TMA producer warp
+// streams 64-wide K blocks of all six slices of the 128 "row" columns and of the 64 "column" columns
+// (SWIZZLE_64B, 3 stages of 72 KB); one thread issues the 42 tcgen05.mma.kind::i8 instructions of a stage into six
+// TMEM accumulators (6 x 64 columns); four epilogue warps read the accumulators back with tcgen05.ld, combine the
+// groups exactly in int64, scale by 2^(41 - sh_i - sh_j) and add into H.
+// Every wait on an mbarrier is bounded; when one expires the CTA records PTQ_ERR_TIMEOUT, drains and returns.
+#pragma once
+#include <cuda.h>
+#include "common.cuh"
+
+namespace ptq {
+
+constexpr int kSlices = 6;
+constexpr int kGroups = 6;                 // groups t = a + b = 0..5
+constexpr int kGramTM = 128;               // tile rows
+constexpr int kGramTN = 64;                // tile columns
+constexpr int kGramKB = 64;                // K block (int8 elements = bytes)
+constexpr int kGramStages = 3;
+constexpr int kGramABytes = kGramTM * kGramKB;                    // 8 KB per slice
+constexpr int kGramBBytes = kGramTN * kGramKB;                    // 4 KB per slice
+constexpr int kGramStageBytes = kSlices * (kGramABytes + kGramBBytes);   // 72 KB
+constexpr int kGramSmemBytes = kGramStages * kGramStageBytes + 1024 /*align*/ + 256 /*barriers*/;
+constexpr int kGramThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM, warps 2..5: epilogue
+constexpr int kGramMaxChunk = 16384;       // calibration columns per launch: 6 * 2^14 * 16384 < 2^31
+constexpr int kShiftTarget = 46;
+
+inline size_t gram_workspace_bytes(int cols, int n) {
+    const size_t cols_pad = (size_t)cdiv(cols, 128) * 128;
+    const int chunk = n < kGramMaxChunk ? n : kGramMaxChunk;
+    const size_t n_pad = (size_t)cdiv(chunk, 128) * 128;
+    return align_up(kSlices * cols_pad * n_pad) + align_up(cols_pad * sizeof(int32_t));
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Slicing pre-pass: one CTA per (padded) row.
+// ------------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) gram_split_kernel(const float* __restrict__ X, int cols, int n, int64_t ldx,
+                                                          int cols_pad, int n_pad, int vec_ok,
+                                                          int8_t* __restrict__ Q, int32_t* __restrict__ shifts,
+                                                          int32_t* status) {
+    __shared__ float smax[256];
+    __shared__ int sbad;
+    const int row = blockIdx.x;
+    const size_t plane = (size_t)cols_pad * n_pad;
+    int8_t* q0 = Q + (size_t)row * n_pad;
+    if (row >= cols) {   // padding rows: zeros
+        for (int k = threadIdx.x * 4; k < n_pad; k += 1024)
+#pragma unroll
+            for (int s = 0; s < kSlices; ++s) *reinterpret_cast<uint32_t*>(q0 + s * plane + k) = 0u;
+        if (threadIdx.x == 0) shifts[row] = 0;
+        return;
+    }
+    if (threadIdx.x == 0) sbad = 0;
+    __syncthreads();
+    const float* x = X + (int64_t)row * ldx;
+    float m = 0.f;
+    bool bad = false;
+    for (int k = threadIdx.x * 4; k < n; k += 1024) {
+        if (vec_ok && k + 3 < n) {
+            const float4 v = *reinterpret_cast<const float4*>(x + k);
+            bad |= !isfinite(v.x) | !isfinite(v.y) | !isfinite(v.z) | !isfinite(v.w);
+            m = fmaxf(m, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
+        } else {
+            for (int kk = k; kk < n; ++kk) { bad |= !isfinite(x[kk]); m = fmaxf(m, fabsf(x[kk])); }
+        }
+    }
+    if (bad) sbad = 1;
+    smax[threadIdx.x] = m;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w) smax[threadIdx.x] = fmaxf(smax[threadIdx.x], smax[threadIdx.x + w]);
+        __syncthreads();
+    }
+    const float rowmax = smax[0];
+    const bool rowbad = sbad != 0;
+    if (rowbad && threadIdx.x == 0) report(status, PTQ_ERR_NONFINITE, row);
+    int sh = 0;
+    if (rowmax > 0.f && !rowbad) sh = kShiftTarget - (ilogbf(rowmax) + 1);   // |x| 2^sh < 2^46
+    if (threadIdx.x == 0) shifts[row] = sh;
+    for (int k = threadIdx.x * 4; k < n_pad; k += 1024) {
+        long long v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int kk = k + u;
+            const float xv = (kk < n && !rowbad) ? x[kk] : 0.f;
+            v[u] = __double2ll_rn(scalbn((double)xv, sh));
+        }
+        uint32_t packed[kSlices];
+#pragma unroll
+        for (int s = 0; s < kSlices; ++s) packed[s] = 0u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            long long t = v[u];
+#pragma unroll
+            for (int s = kSlices - 1; s >= 0; --s) {          // least significant digit first
+                const long long d = ((t + 128) & 255) - 128;  // balanced digit in [-128, 127]
+                t = (t - d) >> 8;
+                packed[s] |= ((uint32_t)(d & 255)) << (8 * u);
+            }
+        }
+#pragma unroll
+        for (int s = 0; s < kSlices; ++s) *reinterpret_cast<uint32_t*>(q0 + s * plane + k) = packed[s];
+    }
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after about a second of polling or as soon as another thread of the CTA gave up.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    const long long t0 = clock64();
+    uint32_t it = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++it & 255u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > 2000000000LL) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tmap, int c0, int c1, int c2,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(tmap), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %5, %5, %5}, p;\n\t}\n"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor: K-major operand, 64-byte rows, SWIZZLE_64B; 8-row groups are 512 bytes apart.
+__device__ __forceinline__ uint64_t make_desc_sw64(uint32_t smem_addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr >> 4) & 0x3FFF);        // start address / 16
+    d |= (uint64_t)1 << 16;                            // leading byte offset / 16 (not used by swizzled K-major)
+    d |= (uint64_t)(512 >> 4) << 32;                   // stride byte offset / 16
+    d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
+    d |= (uint64_t)4 << 61;                            // SWIZZLE_64B
+    return d;
+}
+
+// Instruction descriptor: int8 x int8 -> int32, both operands K-major, M = 128, N = 64.
+constexpr uint32_t kGramIdesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGramTN >> 3) << 17) |
+                                ((uint32_t)(kGramTM >> 4) << 24);
+
+// Tile t of the enumeration: row block bi (128 rows), column block bj (64 columns) with 64*bj + 63 >= 128*bi.
+__device__ __forceinline__ void gram_tile_coords(int tile, int nbj, int& bi, int& bj) {
+    int b = 0, rem = tile;
+    for (;;) {
+        const int cnt = nbj - 2 * b;    // column blocks 2b .. nbj-1
+        if (rem < cnt) break;
+        rem -= cnt;
+        ++b;
+    }
+    bi = b;
+    bj = 2 * b + rem;
+}
+
+__global__ void __launch_bounds__(kGramThreads, 1)
+gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
+               double* __restrict__ H, int cols, int n_pad,
+               const int32_t* __restrict__ shifts, int num_tiles, int nbj, int32_t* status) {
+    extern __shared__ unsigned char gram_smem_raw[];
+    const uint32_t raw = smem_u32(gram_smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    unsigned char* base_ptr = gram_smem_raw + (base - raw);
+    // barriers live after the stages
+    uint64_t* bars = reinterpret_cast<uint64_t*>(base_ptr + kGramStages * kGramStageBytes);
+    const uint32_t bar0 = base + kGramStages * kGramStageBytes;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kGramStages + s); };
+    const uint32_t acc_full = bar0 + 8u * (2 * kGramStages);
+    const uint32_t acc_empty = bar0 + 8u * (2 * kGramStages + 1);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGramStages + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nkb = n_pad / kGramKB;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGramStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+        mbar_init(acc_full, 1);
+        mbar_init(acc_empty, 128);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int armed[kGramStages];
+#pragma unroll
+            for (int s = 0; s < kGramStages; ++s) armed[s] = -1;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                int bi, bj;
+                gram_tile_coords(tile, nbj, bi, bj);
+                for (int kb = 0; kb < nkb && ok; ++kb) {
+                    ok = mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag);
+                    if (!ok) break;
+                    const uint32_t sbase = base + stage * kGramStageBytes;
+                    mbar_arrive_expect_tx(full_bar(stage), kGramStageBytes);
+                    armed[stage] = (int)phase;
+#pragma unroll
+                    for (int s = 0; s < kSlices; ++s) {
+                        tma_load_3d(sbase + s * kGramABytes, &tmapA, kb * kGramKB, bi * kGramTM, s, full_bar(stage));
+                        tma_load_3d(sbase + kSlices * kGramABytes + s * kGramBBytes, &tmapB, kb * kGramKB,
+                                    bj * kGramTN, s, full_bar(stage));
+                    }
+                    if (++stage == kGramStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // drain: wait (bounded) until the copies already issued have landed
+                for (int s = 0; s < kGramStages; ++s)
+                    if (armed[s] >= 0) {
+                        const long long t0 = clock64();
+                        while (!mbar_try_wait(full_bar(s), (uint32_t)armed[s]) && clock64() - t0 < 200000000LL) {}
+                    }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                ok = mbar_wait_bounded(acc_empty, acc_phase ^ 1u, abort_flag);   // epilogue has drained TMEM
+                if (!ok) break;
+                tc_fence_after();
+                for (int kb = 0; kb < nkb && ok; ++kb) {
+                    ok = mbar_wait_bounded(full_bar(stage), phase, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sbase = base + stage * kGramStageBytes;
+#pragma unroll
+                    for (int t = 0; t < kGroups; ++t) {
+#pragma unroll
+                        for (int a = 0; a <= t; ++a) {
+                            const int b = t - a;
+                            const uint64_t ad = make_desc_sw64(sbase + a * kGramABytes);
+                            const uint64_t bd = make_desc_sw64(sbase + kSlices * kGramABytes + b * kGramBBytes);
+#pragma unroll
+                            for (int ks = 0; ks < kGramKB / 32; ++ks) {
+                                const uint32_t acc = (kb > 0 || a > 0 || ks > 0) ? 1u : 0u;
+                                tc_mma_i8(tmem_base + t * kGramTN, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 2),
+                                          kGramIdesc, acc);
+                            }
+                        }
+                    }
+                    tc_commit(empty_bar(stage));     // the stage may be refilled once these MMAs have read it
+                    if (++stage == kGramStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) tc_commit(acc_full);         // accumulators complete
+                acc_phase ^= 1u;
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue (warps 2..5)
+        const int quarter = warp & 3;                 // TMEM lanes this warp may read
+        const int r_in_tile = quarter * 32 + lane;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            int bi, bj;
+            gram_tile_coords(tile, nbj, bi, bj);
+            ok = mbar_wait_bounded(acc_full, acc_phase, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int row = bi * kGramTM + r_in_tile;
+            const int sh_i = row < cols ? shifts[row] : 0;
+#pragma unroll 1
+            for (int ch = 0; ch < kGramTN / 16; ++ch) {
+                long long lo[16], hi[16];
+                uint32_t r[16];
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + ch * 16;
+                // groups 5, 4, 3 -> lo = G5 + 2^8 G4 + 2^16 G3 ; groups 2, 1, 0 -> hi = G2 + 2^8 G1 + 2^16 G0
+                tc_ld16(taddr + 5 * kGramTN, r); tc_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) lo[c] = (long long)(int)r[c];
+                tc_ld16(taddr + 4 * kGramTN, r); tc_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) lo[c] += (long long)(int)r[c] << 8;
+                tc_ld16(taddr + 3 * kGramTN, r); tc_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) lo[c] += (long long)(int)r[c] << 16;
+                tc_ld16(taddr + 2 * kGramTN, r); tc_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) hi[c] = (long long)(int)r[c];
+                tc_ld16(taddr + 1 * kGramTN, r); tc_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) hi[c] += (long long)(int)r[c] << 8;
+                tc_ld16(taddr + 0 * kGramTN, r); tc_wait_ld();
+#pragma unroll
+                for (int c = 0; c < 16; ++c) hi[c] += (long long)(int)r[c] << 16;
+                if (row < cols) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const int col = bj * kGramTN + ch * 16 + c;
+                        if (col < cols) {
+                            const double v = fma((double)hi[c], 16777216.0, (double)lo[c]);
+                            const int e = 41 - sh_i - shifts[col];
+                            const double add = scalbn(v, e);
+                            // tiles that straddle the diagonal hold both (i, j) and (j, i): each writes itself only
+                            const bool straddle = (bj * kGramTN < bi * kGramTM + kGramTM);
+                            const double out = H[(int64_t)row * cols + col] + add;
+                            H[(int64_t)row * cols + col] = out;
+                            if (!straddle) H[(int64_t)col * cols + row] = out;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty);
+            acc_phase ^= 1u;
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+    if (threadIdx.x == 0 && *abort_flag) report(status, PTQ_ERR_TIMEOUT, blockIdx.x);
+}
+
+// ------------------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn get_encode_tiled() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+inline int make_slice_map(CUtensorMap* m, int8_t* Q, int cols_pad, int n_pad, int box_rows) {
+    EncodeTiledFn enc = get_encode_tiled();
+    if (!enc) return PTQ_ERR_CUDA;
+    const cuuint64_t dims[3] = {(cuuint64_t)n_pad, (cuuint64_t)cols_pad, (cuuint64_t)kSlices};
+    const cuuint64_t strides[2] = {(cuuint64_t)n_pad, (cuuint64_t)cols_pad * (cuuint64_t)n_pad};
+    const cuuint32_t box[3] = {(cuuint32_t)kGramKB, (cuuint32_t)box_rows, 1u};
+    const cuuint32_t estr[3] = {1u, 1u, 1u};
+    const CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, Q, dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? PTQ_OK : PTQ_ERR_CUDA;
+}
+
+inline int gram_accumulate(double* H, const float* X, int cols, int n, int64_t ldx, void* ws, int32_t* status,
+                           cudaStream_t stream) {
+    static bool attr_done = false;
+    static int num_sms = 0;
+    if (!attr_done) {
+        if (cudaFuncSetAttribute(gram_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGramSmemBytes) !=
+            cudaSuccess)
+            return PTQ_ERR_CUDA;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+        attr_done = true;
+    }
+    const int cols_pad = cdiv(cols, 128) * 128;
+    const int max_chunk = n < kGramMaxChunk ? n : kGramMaxChunk;
+    const size_t n_pad_max = (size_t)cdiv(max_chunk, 128) * 128;
+    Carver cv(ws);
+    int8_t* Q = cv.take<int8_t>(kSlices * (size_t)cols_pad * n_pad_max);
+    int32_t* shifts = cv.take<int32_t>(cols_pad);
+    const int nbi = cdiv(cols, kGramTM), nbj = cdiv(cols, kGramTN);
+    int num_tiles = 0;
+    for (int b = 0; b < nbi; ++b) num_tiles += (nbj - 2 * b) > 0 ? (nbj - 2 * b) : 0;
+    for (int c0 = 0; c0 < n; c0 += kGramMaxChunk) {
+        const int nc = n - c0 < kGramMaxChunk ? n - c0 : kGramMaxChunk;
+        const int n_pad = cdiv(nc, 128) * 128;
+        const int vec_ok = (aligned16(X) && (ldx & 3) == 0) ? 1 : 0;
+        gram_split_kernel<<<cols_pad, 256, 0, stream>>>(X + c0, cols, nc, ldx, cols_pad, n_pad, vec_ok, Q, shifts,
+                                                        status);
+        CUtensorMap mapA, mapB;
+        int st = make_slice_map(&mapA, Q, cols_pad, n_pad, kGramTM);
+        if (st) return st;
+        st = make_slice_map(&mapB, Q, cols_pad, n_pad, kGramTN);
+        if (st) return st;
+        const int grid = num_tiles < num_sms ? num_tiles : num_sms;
+        gram_i8_kernel<<<grid, kGramThreads, kGramSmemBytes, stream>>>(mapA, mapB, H, cols, n_pad, shifts, num_tiles,
+                                                                     nbj, status);
+        if (cudaGetLastError() != cudaSuccess) return PTQ_ERR_CUDA;
+    }
+    return PTQ_OK;
+}
+
+}  // namespace ptq

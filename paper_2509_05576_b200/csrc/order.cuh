@@ -1,0 +1,128 @@
+// Grid helper, column sensitivity scores and the stable descending column order (Sec. 4.2 steps 1-3).
+#pragma once
+#include "common.cuh"
+
+namespace ptq {
+
+// quant(): nearest level of the per-row grid, ties to even, clamped to the code range (all in float64).
+__device__ __forceinline__ double quant_code_d(double w, double sc, double zp, double maxq) {
+    double c = rint(w / sc) + zp;
+    c = fmax(c, 0.0);
+    c = fmin(c, maxq);
+    return c;
+}
+
+// One CTA per row: lo = min(min_j w, 0), hi = max(max_j w, 0); scale = (hi - lo) / (2^bits - 1); zero = rint(-lo / scale).
+__global__ void __launch_bounds__(256) minmax_grid_kernel(const float* __restrict__ W, int rows, int cols, int64_t ldw,
+                                                           int bits, float* __restrict__ scale,
+                                                           float* __restrict__ zero, int32_t* status) {
+    __shared__ float slo[256], shi[256];
+    __shared__ int sbad;
+    const int i = blockIdx.x;
+    if (threadIdx.x == 0) sbad = 0;
+    __syncthreads();
+    float lo = 0.f, hi = 0.f;
+    bool bad = false;
+    for (int j = threadIdx.x; j < cols; j += 256) {
+        const float w = W[(int64_t)i * ldw + j];
+        if (!isfinite(w)) bad = true;
+        lo = fminf(lo, w);
+        hi = fmaxf(hi, w);
+    }
+    if (bad) sbad = 1;
+    slo[threadIdx.x] = lo;
+    shi[threadIdx.x] = hi;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+        if (threadIdx.x < s) {
+            slo[threadIdx.x] = fminf(slo[threadIdx.x], slo[threadIdx.x + s]);
+            shi[threadIdx.x] = fmaxf(shi[threadIdx.x], shi[threadIdx.x + s]);
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (sbad) report(status, PTQ_ERR_NONFINITE, i);
+        const double l = (double)slo[0], h = (double)shi[0];
+        if (h == l) {
+            scale[i] = 1.0f;
+            zero[i] = 0.0f;
+        } else {
+            const double s = (h - l) / (double)((1 << bits) - 1);
+            scale[i] = (float)s;
+            zero[i] = (float)rint(-l / s);
+        }
+    }
+}
+
+constexpr int kScoreRowChunk = 64;
+
+// partial[ch][j] = sum over the rows of chunk ch (ascending) of the score numerator of w_ij.
+__global__ void __launch_bounds__(128) score_partial_kernel(const float* __restrict__ W, int rows, int cols,
+                                                             int64_t ldw, const float* __restrict__ scale,
+                                                             const float* __restrict__ zero, int bits, int mode,
+                                                             double* __restrict__ partial) {
+    const int j = blockIdx.x * 128 + threadIdx.x;
+    const int ch = blockIdx.y;
+    if (j >= cols) return;
+    const int r0 = ch * kScoreRowChunk;
+    const int r1 = min(rows, r0 + kScoreRowChunk);
+    const double maxq = (double)((1 << bits) - 1);
+    const bool use_err = (mode == PTQ_SCORE_QERR || mode == PTQ_SCORE_ERR);
+    double s = 0.0;
+    for (int i = r0; i < r1; ++i) {
+        const double w = (double)W[(int64_t)i * ldw + j];
+        if (use_err) {
+            const double sc = (double)scale[i], zp = (double)zero[i];
+            const double q = sc * (quant_code_d(w, sc, zp, maxq) - zp);
+            const double d = w - q;
+            s = fma(d, d, s);
+        } else {
+            s = fma(w, w, s);
+        }
+    }
+    partial[(int64_t)ch * cols + j] = s;
+}
+
+// S_j = (sum of the chunk partials, ascending) / (2 [Hinv]_jj)  for the sensitivity modes.
+__global__ void __launch_bounds__(128) score_final_kernel(const double* __restrict__ partial, int chunks, int cols,
+                                                           const double* __restrict__ hinv_diag, int mode,
+                                                           double* __restrict__ S, int32_t* status) {
+    const int j = blockIdx.x * 128 + threadIdx.x;
+    if (j >= cols) return;
+    double s = 0.0;
+    if (mode != PTQ_SCORE_NONE) {
+        for (int ch = 0; ch < chunks; ++ch) s += partial[(int64_t)ch * cols + j];
+        if (mode == PTQ_SCORE_QERR || mode == PTQ_SCORE_PRUNE) s = s / (2.0 * hinv_diag[j]);
+    }
+    if (!isfinite(s)) report(status, PTQ_ERR_NONFINITE, j);
+    S[j] = s;
+}
+
+// Order-preserving map from float64 to uint64 (total order, so even non-finite scores give a permutation).
+__device__ __forceinline__ unsigned long long sortable_key(double x) {
+    unsigned long long u = (unsigned long long)__double_as_longlong(x);
+    return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
+}
+
+// perm[rank_j] = j with rank_j = #{k : S_k > S_j, or S_k == S_j and k < j}: a stable descending sort by counting.
+__global__ void __launch_bounds__(256) rank_sort_kernel(const double* __restrict__ S, int cols,
+                                                         int32_t* __restrict__ perm) {
+    __shared__ unsigned long long keys[256];
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    const unsigned long long kj = j < cols ? sortable_key(S[j]) : 0ull;
+    int rank = 0;
+    for (int t0 = 0; t0 < cols; t0 += 256) {
+        const int k = t0 + threadIdx.x;
+        keys[threadIdx.x] = k < cols ? sortable_key(S[k]) : 0ull;
+        __syncthreads();
+        const int lim = min(256, cols - t0);
+        for (int t = 0; t < lim; ++t) {
+            const unsigned long long kk = keys[t];
+            rank += (kk > kj || (kk == kj && (t0 + t) < j)) ? 1 : 0;
+        }
+        __syncthreads();
+    }
+    if (j < cols) perm[rank] = j;
+}
+
+}  // namespace ptq

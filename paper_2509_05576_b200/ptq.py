@@ -1,0 +1,234 @@
+"""Thin binding over the C-ABI CUDA library ``libptq.so`` (declared in ``include/ptq.h``).
+
+Only argument marshalling happens here: every step of the path runs in the library's kernels.
+torch is used for device memory and streams.  There is no CPU fallback: if the library is missing
+or no CUDA device is present, the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_double, c_int, c_int64, c_size_t, c_void_p
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libptq.so")
+
+OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_NOT_SPD, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA, ERR_UNSUPPORTED = range(9)
+DAMP_REL_MEAN_DIAG, DAMP_ABS = 0, 1
+SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
+CALL_HESSIAN_ACCUMULATE, CALL_PREPARE_HINV, CALL_SENSITIVITY_ORDER, CALL_QUANTIZE_LAYER, CALL_HESSIAN_ACCUMULATE_F64 = range(5)
+
+EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
+           "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_quantize_layer", "ptq_status_string", "ptq_version"]
+
+
+class PtqError(RuntimeError):
+    def __init__(self, code, where, index=None):
+        msg = f"{where}: {status_string(code)} (status {code})"
+        if index is not None:
+            msg += f", index {index}"
+        super().__init__(msg)
+        self.code = code
+        self.index = index
+
+
+_lib = None
+
+
+def lib():
+    """Loads ``libptq.so`` (built in-tree by ``paper_2509_05576_b200.build``); raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2509_05576_b200.build` "
+                               "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp = c_void_p
+        L.ptq_workspace_bytes.argtypes = [c_int, c_int, c_int, c_int]
+        L.ptq_workspace_bytes.restype = c_size_t
+        for name in ("ptq_hessian_accumulate", "ptq_hessian_accumulate_f64"):
+            getattr(L, name).argtypes = [vp, vp, c_int, c_int, c_int64, vp, c_size_t, vp, vp]
+        L.ptq_prepare_hinv.argtypes = [vp, c_int, c_int, c_double, vp, vp, vp, vp, c_size_t, vp, vp]
+        L.ptq_minmax_grid.argtypes = [vp, c_int, c_int, c_int64, c_int, vp, vp, vp, vp]
+        L.ptq_sensitivity_order.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, c_size_t,
+                                            vp, vp]
+        L.ptq_quantize_layer.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, vp, c_int, vp, vp, vp, vp, vp,
+                                         c_size_t, vp, vp]
+        L.ptq_status_string.argtypes = [c_int]
+        L.ptq_status_string.restype = ctypes.c_char_p
+        L.ptq_version.restype = c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().ptq_status_string(int(code)).decode()
+
+
+def workspace_bytes(call_id: int, rows: int, cols: int, n: int) -> int:
+    return int(lib().ptq_workspace_bytes(int(call_id), int(rows), int(cols), int(n)))
+
+
+def _ptr(t):
+    return None if t is None else c_void_p(t.data_ptr())
+
+
+def _stream(stream):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return c_void_p(s.cuda_stream)
+
+
+def _dev(t, dtype, name):
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (the library has no CPU path)")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}")
+    return t
+
+
+def _rowmajor(t, name):
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError(f"{name} must be 2-D with unit column stride")
+    return t.stride(0)
+
+
+class Workspace:
+    """A growable device scratch buffer handed to the library calls."""
+
+    def __init__(self, device="cuda"):
+        self.device = torch.device(device)
+        self.buf = None
+
+    def get(self, nbytes: int):
+        if self.buf is None or self.buf.numel() < nbytes:
+            self.buf = None
+            self.buf = torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=self.device)
+        return self.buf
+
+
+def new_status(device="cuda"):
+    return torch.zeros(4, dtype=torch.int32, device=device)
+
+
+def check_status(status, where="ptq"):
+    """Synchronises and raises if a kernel recorded an error in the status word."""
+    code, index, aux, _ = status.cpu().tolist()
+    if code != OK:
+        raise PtqError(code, where, index)
+
+
+def _check(ret, where):
+    if ret != OK:
+        raise PtqError(ret, where)
+
+
+def hessian_accumulate(H, X, ws, status, stream=None, f64=False):
+    """H += 2 X X^T (Sec. 3).  H [cols, cols] float64, X [cols, n] float32, both on the device."""
+    _dev(H, torch.float64, "H"); _dev(X, torch.float32, "X")
+    cols, n = X.shape
+    ldx = _rowmajor(X, "X")
+    if H.shape != (cols, cols) or not H.is_contiguous():
+        raise ValueError("H must be contiguous [cols, cols]")
+    fn = lib().ptq_hessian_accumulate_f64 if f64 else lib().ptq_hessian_accumulate
+    need = workspace_bytes(CALL_HESSIAN_ACCUMULATE_F64 if f64 else CALL_HESSIAN_ACCUMULATE, 0, cols, n)
+    buf = ws.get(need)
+    _check(fn(_ptr(H), _ptr(X), cols, n, ldx, _ptr(buf), buf.numel(), _ptr(status), _stream(stream)),
+           "ptq_hessian_accumulate")
+
+
+def prepare_hinv(H, damp, damp_mode, Hinv, Hinv_diag, lambda_out, ws, status, stream=None):
+    """Hinv = (H + lambda I)^-1 (Sec. 5 item 1); also its diagonal and lambda (device scalars)."""
+    _dev(H, torch.float64, "H"); _dev(Hinv, torch.float64, "Hinv")
+    cols = H.shape[0]
+    buf = ws.get(workspace_bytes(CALL_PREPARE_HINV, 0, cols, 0))
+    _check(lib().ptq_prepare_hinv(_ptr(H), cols, int(damp_mode), float(damp), _ptr(Hinv), _ptr(Hinv_diag),
+                                  _ptr(lambda_out), _ptr(buf), buf.numel(), _ptr(status), _stream(stream)),
+           "ptq_prepare_hinv")
+
+
+def minmax_grid(W, bits, scale, zero, status, stream=None):
+    _dev(W, torch.float32, "W")
+    rows, cols = W.shape
+    _check(lib().ptq_minmax_grid(_ptr(W), rows, cols, _rowmajor(W, "W"), int(bits), _ptr(scale), _ptr(zero),
+                                 _ptr(status), _stream(stream)), "ptq_minmax_grid")
+
+
+def sensitivity_order(W, Hinv_diag, scale, zero, bits, score_mode, S, perm, ws, status, stream=None):
+    """Sec. 4.2 steps 1-3: column scores S and the descending, stable column order perm."""
+    _dev(W, torch.float32, "W")
+    rows, cols = W.shape
+    buf = ws.get(workspace_bytes(CALL_SENSITIVITY_ORDER, rows, cols, 0))
+    _check(lib().ptq_sensitivity_order(_ptr(W), rows, cols, _rowmajor(W, "W"), _ptr(Hinv_diag), _ptr(scale),
+                                       _ptr(zero), int(bits), int(score_mode), _ptr(S), _ptr(perm), _ptr(buf),
+                                       buf.numel(), _ptr(status), _stream(stream)), "ptq_sensitivity_order")
+
+
+def quantize_layer(W, Hinv, perm, scale, zero, bits, codes, What, H_undamped, loss_out, ws, status, stream=None):
+    """Sec. 4.2 steps 3-5 (Eq. 11, Eq. 12): the column-synchronous sweep.  Outputs in original column order."""
+    _dev(W, torch.float32, "W"); _dev(Hinv, torch.float64, "Hinv"); _dev(perm, torch.int32, "perm")
+    _dev(codes, torch.uint8, "codes")
+    rows, cols = W.shape
+    buf = ws.get(workspace_bytes(CALL_QUANTIZE_LAYER, rows, cols, 0))
+    _check(lib().ptq_quantize_layer(_ptr(W), rows, cols, _rowmajor(W, "W"), _ptr(Hinv), _ptr(perm), _ptr(scale),
+                                    _ptr(zero), int(bits), _ptr(codes), _ptr(What), _ptr(H_undamped), _ptr(loss_out),
+                                    _ptr(buf), buf.numel(), _ptr(status), _stream(stream)), "ptq_quantize_layer")
+
+
+class LayerBuffers:
+    """Device outputs and scratch of one layer shape, allocated once and reused across calls."""
+
+    def __init__(self, rows, cols, device="cuda"):
+        d = torch.device(device)
+        self.rows, self.cols = rows, cols
+        self.H = torch.empty((cols, cols), dtype=torch.float64, device=d)
+        self.Hinv = torch.empty((cols, cols), dtype=torch.float64, device=d)
+        self.Hinv_diag = torch.empty(cols, dtype=torch.float64, device=d)
+        self.lam = torch.empty(1, dtype=torch.float64, device=d)
+        self.scale = torch.empty(rows, dtype=torch.float32, device=d)
+        self.zero = torch.empty(rows, dtype=torch.float32, device=d)
+        self.S = torch.empty(cols, dtype=torch.float64, device=d)
+        self.perm = torch.empty(cols, dtype=torch.int32, device=d)
+        self.codes = torch.empty((rows, cols), dtype=torch.uint8, device=d)
+        self.What = torch.empty((rows, cols), dtype=torch.float32, device=d)
+        self.loss = torch.empty(1, dtype=torch.float64, device=d)
+        self.status = new_status(d)
+
+
+def quantize_layer_full(W, X, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG, score_mode=SCORE_QERR, bufs=None, ws=None,
+                        stream=None, want_loss=True, events=None, gram_f64=False):
+    """The whole hot path on one layer (all device-side, asynchronous on the stream):
+    Hessian -> damped inverse -> grid -> scores + order -> column sweep -> codes, What, loss.
+
+    ``events``: optional list receiving (stage name, start event, end event) for per-stage timing.
+    Returns the LayerBuffers holding the outputs; call ``check_status(bufs.status)`` after synchronising.
+    """
+    rows, cols = W.shape
+    bufs = bufs or LayerBuffers(rows, cols, W.device)
+    ws = ws or Workspace(W.device)
+    st = bufs.status
+    s = torch.cuda.current_stream() if stream is None else stream
+
+    def timed(name, fn):
+        if events is None:
+            fn()
+            return
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(s)
+        fn()
+        b.record(s)
+        events.append((name, a, b))
+
+    with torch.cuda.stream(s):
+        st.zero_()
+        bufs.H.zero_()
+        timed("hessian", lambda: hessian_accumulate(bufs.H, X, ws, st, s, f64=gram_f64))
+        timed("inverse", lambda: prepare_hinv(bufs.H, damp, damp_mode, bufs.Hinv, bufs.Hinv_diag, bufs.lam, ws, st, s))
+        timed("grid", lambda: minmax_grid(W, bits, bufs.scale, bufs.zero, st, s))
+        timed("order", lambda: sensitivity_order(W, bufs.Hinv_diag, bufs.scale, bufs.zero, bits, score_mode, bufs.S,
+                                                 bufs.perm, ws, st, s))
+        timed("sweep", lambda: quantize_layer(W, bufs.Hinv, bufs.perm, bufs.scale, bufs.zero, bits, bufs.codes,
+                                              bufs.What, bufs.H if want_loss else None,
+                                              bufs.loss if want_loss else None, ws, st, s))
+    return bufs

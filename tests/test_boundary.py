@@ -1,0 +1,85 @@
+"""CPU-side checks of the C-ABI boundary: the library loads, exports every symbol the header declares, sizes its
+workspaces sanely and rejects bad arguments on the host before anything is launched (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2509_05576_b200 import build as ptq_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    path = ptq_build.build()
+    from paper_2509_05576_b200 import ptq
+    assert ptq.LIB_PATH == path
+    return ptq.lib()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ptq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ptq_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared()
+    assert {"ptq_hessian_accumulate", "ptq_prepare_hinv", "ptq_sensitivity_order", "ptq_quantize_layer"} <= set(names)
+    for name in names:
+        assert hasattr(lib, name), f"{name} is declared in ptq.h but not exported"
+    from paper_2509_05576_b200 import ptq
+    assert sorted(ptq.EXPORTS) == names
+    assert lib.ptq_version() >= 1
+    assert ptq.status_string(4) == "matrix not positive definite"
+
+
+def test_workspace_sizes(lib):
+    from paper_2509_05576_b200 import ptq
+    for call in range(5):
+        small = ptq.workspace_bytes(call, 64, 128, 1024)
+        big = ptq.workspace_bytes(call, 256, 2304, 4096)
+        assert 0 < small < big
+        assert small % 256 == 0
+    # the inverse needs two cols x cols float64 matrices
+    assert ptq.workspace_bytes(ptq.CALL_PREPARE_HINV, 0, 2304, 0) == 2 * 2304 * 2304 * 8
+    assert ptq.workspace_bytes(99, 1, 1, 1) == 0
+    # largest benchmark shape stays far below the 180 GB of one GPU
+    total = sum(ptq.workspace_bytes(c, 4096, 11008, 8192) for c in range(4))
+    assert total < 8 * 2 ** 30
+
+
+def test_bad_arguments_are_rejected_on_the_host(lib):
+    from paper_2509_05576_b200 import ptq
+    vp = ctypes.c_void_p
+    fake = vp(4096)          # never dereferenced: argument checks come first
+    odd = vp(4100)           # not 16-byte aligned
+    assert lib.ptq_hessian_accumulate(None, fake, 8, 8, 8, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_hessian_accumulate(fake, fake, 8, 16, 8, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG  # ldx < n
+    assert lib.ptq_hessian_accumulate(odd, fake, 8, 8, 8, fake, 1 << 30, fake, None) == ptq.ERR_ALIGNMENT
+    assert lib.ptq_hessian_accumulate(fake, fake, 8, 8, 8, fake, 16, fake, None) == ptq.ERR_WORKSPACE
+    assert lib.ptq_hessian_accumulate_f64(fake, fake, 0, 8, 8, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_prepare_hinv(fake, 8, 7, 0.01, fake, fake, fake, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_prepare_hinv(fake, 8, 0, -1.0, fake, fake, fake, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_prepare_hinv(fake, 8, 0, 0.01, fake, fake, fake, fake, 8, fake, None) == ptq.ERR_WORKSPACE
+    assert lib.ptq_minmax_grid(fake, 4, 8, 8, 9, fake, fake, fake, None) == ptq.ERR_INVALID_ARG      # bits > 8
+    assert lib.ptq_minmax_grid(fake, 4, 8, 4, 4, fake, fake, fake, None) == ptq.ERR_INVALID_ARG      # ldw < cols
+    assert lib.ptq_sensitivity_order(fake, 4, 8, 8, None, fake, fake, 4, 0, fake, fake, fake, 1 << 30, fake,
+                                     None) == ptq.ERR_INVALID_ARG                                   # QERR needs diag
+    assert lib.ptq_sensitivity_order(fake, 4, 8, 8, fake, fake, fake, 4, 5, fake, fake, fake, 1 << 30, fake,
+                                     None) == ptq.ERR_INVALID_ARG                                   # unknown mode
+    assert lib.ptq_quantize_layer(fake, 4, 8, 8, fake, None, fake, fake, 4, fake, None, None, None, fake, 1 << 30,
+                                  fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_quantize_layer(fake, 4, 8, 8, fake, fake, fake, fake, 1, fake, None, None, None, fake, 1 << 30,
+                                  fake, None) == ptq.ERR_INVALID_ARG                                # bits < 2
+    assert lib.ptq_quantize_layer(fake, 4, 8, 8, fake, fake, fake, fake, 4, fake, None, None, None, fake, 64,
+                                  fake, None) == ptq.ERR_WORKSPACE
+
+
+def test_binding_refuses_cpu_tensors(lib):
+    import torch
+    from paper_2509_05576_b200 import ptq
+    with pytest.raises(ValueError):
+        ptq.hessian_accumulate(torch.zeros(4, 4, dtype=torch.float64), torch.zeros(4, 8), None, None)

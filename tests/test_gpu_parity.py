@@ -1,0 +1,267 @@
+"""GPU parity tests: every stage and the whole path, through the C-ABI library, against the CPU oracle on the
+same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_05576_b200 import ptq
+from paper_2509_05576_b200 import workloads as wl
+from parity import (assert_layer_parity, compare_codes, gpu_layer, oracle_layer, LOSS_RTOL, WHAT_RTOL)
+
+pytestmark = pytest.mark.gpu
+
+
+def _layer(rows, cols, n, seed, bits=4, xdist="halfnormal", wdist="kaiming"):
+    return wl.make_layer(wl.LayerSpec("t", rows, cols, n, bits, wdist, xdist, seed))
+
+
+def _cuda(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+# ------------------------------------------------------------------------------------------ Hessian
+@pytest.mark.parametrize("cols,n", [(128, 1024), (147, 200), (64, 64), (200, 520), (333, 4096), (32, 36)])
+@pytest.mark.parametrize("f64", [False, True])
+def test_hessian_matches_oracle(cols, n, f64):
+    _, X = _layer(4, cols, n, 100 + cols)
+    ref = oracle.hessian_accumulate(X)
+    H = torch.zeros((cols, cols), dtype=torch.float64, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.hessian_accumulate(H, _cuda(X), ws, st, f64=f64)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    Hn = H.cpu().numpy()
+    assert np.array_equal(Hn, Hn.T)
+    assert np.max(np.abs(Hn - ref)) <= 2e-12 * np.max(np.abs(ref))
+
+
+@pytest.mark.parametrize("xdist", ["normal", "silu", "halfnormal_sparse30"])
+def test_hessian_signed_and_sparse_inputs_accumulate_in_chunks(xdist):
+    cols, n = 190, 768
+    _, X = _layer(4, cols, n, 7, xdist=xdist)
+    X[5] = 0.0                      # a dead input channel
+    X[9] *= 1e-6                    # rows of very different magnitude
+    X[11] *= 3e4
+    ref = oracle.hessian_accumulate(X)
+    H = torch.zeros((cols, cols), dtype=torch.float64, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    Xd = _cuda(X)
+    ptq.hessian_accumulate(H, Xd[:, :256], ws, st)       # strided views: ldx = 768
+    ptq.hessian_accumulate(H, Xd[:, 256:], ws, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    Hn = H.cpu().numpy()
+    scale = np.sqrt(np.outer(np.diag(ref), np.diag(ref))) + 1e-300
+    assert np.max(np.abs(Hn - ref) / scale) <= 1e-11
+    assert np.all(Hn[5] == 0) and np.all(Hn[:, 5] == 0)
+
+
+def test_hessian_reports_nonfinite_input():
+    _, X = _layer(4, 64, 128, 8)
+    X[3, 17] = np.inf
+    H = torch.zeros((64, 64), dtype=torch.float64, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.hessian_accumulate(H, _cuda(X), ws, st)
+    torch.cuda.synchronize()
+    with pytest.raises(ptq.PtqError) as ei:
+        ptq.check_status(st)
+    assert ei.value.code == ptq.ERR_NONFINITE and ei.value.index == 3
+
+
+# ------------------------------------------------------------------------------------------ damped inverse
+@pytest.mark.parametrize("cols,n", [(64, 256), (100, 300), (128, 1024), (257, 200), (600, 700)])
+def test_inverse_matches_oracle(cols, n):
+    _, X = _layer(4, cols, n, 200 + cols)
+    H = oracle.hessian_accumulate(X)
+    ref, ref_diag, ref_lam = oracle.prepare_hinv(H, 0.01, oracle.DAMP_REL_MEAN_DIAG)
+    Hd = _cuda(H)
+    Hinv = torch.empty_like(Hd)
+    diag = torch.empty(cols, dtype=torch.float64, device="cuda")
+    lam = torch.empty(1, dtype=torch.float64, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.prepare_hinv(Hd, 0.01, ptq.DAMP_REL_MEAN_DIAG, Hinv, diag, lam, ws, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    G = Hinv.cpu().numpy()
+    assert abs(lam.item() - ref_lam) <= 1e-14 * ref_lam
+    cond = np.linalg.cond(H + ref_lam * np.eye(cols))
+    assert np.max(np.abs(G - ref)) <= 1e-15 * cond * np.max(np.abs(ref)) * 20
+    assert np.array_equal(G, G.T)
+    assert np.array_equal(diag.cpu().numpy(), np.diag(G))
+    assert np.max(np.abs(np.diag(G) - ref_diag) / ref_diag) <= 1e-15 * cond * 20
+    assert torch.equal(Hd, _cuda(H)), "input H must not be modified"
+
+
+def test_inverse_absolute_damping_and_not_spd_status():
+    _, X = _layer(4, 70, 30, 9)       # rank 30 < 70
+    H = oracle.hessian_accumulate(X)
+    ref, _, _ = oracle.prepare_hinv(H, 0.1, oracle.DAMP_ABS)
+    Hd = _cuda(H)
+    Hinv = torch.empty_like(Hd)
+    diag = torch.empty(70, dtype=torch.float64, device="cuda")
+    lam = torch.empty(1, dtype=torch.float64, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.prepare_hinv(Hd, 0.1, ptq.DAMP_ABS, Hinv, diag, lam, ws, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    assert lam.item() == 0.1
+    assert np.max(np.abs(Hinv.cpu().numpy() - ref)) <= 1e-9 * np.max(np.abs(ref))
+    # not positive definite: reported through the status word, nothing traps
+    bad = _cuda(-np.eye(70))
+    st2 = ptq.new_status()
+    ptq.prepare_hinv(bad, 0.0, ptq.DAMP_ABS, Hinv, diag, lam, ws, st2)
+    torch.cuda.synchronize()
+    with pytest.raises(ptq.PtqError) as ei:
+        ptq.check_status(st2)
+    assert ei.value.code == ptq.ERR_NOT_SPD and ei.value.index == 0
+
+
+# ------------------------------------------------------------------------------------------ grid, scores, order
+@pytest.mark.parametrize("bits", [2, 3, 4, 8])
+def test_grid_is_bit_exact(bits):
+    W, _ = _layer(70, 333, 8, 300 + bits)
+    W[5] = np.abs(W[5]); W[6] = 0.0; W[7] = -np.abs(W[7])
+    ref_s, ref_z = oracle.minmax_grid(W, bits)
+    scale = torch.empty(70, dtype=torch.float32, device="cuda")
+    zero = torch.empty(70, dtype=torch.float32, device="cuda")
+    st = ptq.new_status()
+    ptq.minmax_grid(_cuda(W), bits, scale, zero, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    assert np.array_equal(scale.cpu().numpy(), ref_s) and np.array_equal(zero.cpu().numpy(), ref_z)
+
+
+@pytest.mark.parametrize("mode", [ptq.SCORE_QERR, ptq.SCORE_PRUNE, ptq.SCORE_ERR, ptq.SCORE_W, ptq.SCORE_NONE])
+@pytest.mark.parametrize("rows,cols", [(70, 333), (200, 64), (1, 5)])
+def test_scores_and_order_match_oracle(mode, rows, cols):
+    W, X = _layer(rows, cols, 400, 400 + rows)
+    if cols > 20:
+        W[:, 17] = W[:, 3]              # exact ties must keep the lower index first
+    _, diag, _ = oracle.prepare_hinv(oracle.hessian_accumulate(X))
+    if cols > 20:
+        diag[17] = diag[3]
+    sc, zp = oracle.minmax_grid(W, 4)
+    ref_S, ref_perm = oracle.sensitivity_order(W, diag, sc, zp, 4, mode)
+    S = torch.empty(cols, dtype=torch.float64, device="cuda")
+    perm = torch.empty(cols, dtype=torch.int32, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.sensitivity_order(_cuda(W), _cuda(diag), _cuda(sc), _cuda(zp), 4, mode, S, perm, ws, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    assert np.allclose(S.cpu().numpy(), ref_S, rtol=1e-13, atol=0)
+    assert np.array_equal(perm.cpu().numpy(), ref_perm)
+
+
+# ------------------------------------------------------------------------------------------ column sweep
+def _sweep(W, Hinv, perm, sc, zp, bits, H=None):
+    rows, cols = W.shape
+    codes = torch.empty((rows, cols), dtype=torch.uint8, device="cuda")
+    What = torch.empty((rows, cols), dtype=torch.float32, device="cuda")
+    loss = torch.zeros(1, dtype=torch.float64, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.quantize_layer(_cuda(W), _cuda(Hinv), _cuda(perm), _cuda(sc), _cuda(zp), bits, codes, What,
+                       None if H is None else _cuda(H), None if H is None else loss, ws, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    return codes.cpu().numpy(), What.cpu().numpy(), loss.item()
+
+
+@pytest.mark.parametrize("rows,cols,n,bits", [(64, 128, 1024, 4), (37, 147, 300, 4), (70, 200, 150, 3),
+                                              (33, 64, 100, 8), (5, 9, 30, 2), (130, 321, 512, 4)])
+def test_sweep_matches_oracle_on_identical_inputs(rows, cols, n, bits):
+    W, X = _layer(rows, cols, n, 500 + cols)
+    H = oracle.hessian_accumulate(X)
+    Hinv, diag, _ = oracle.prepare_hinv(H)
+    sc, zp = oracle.minmax_grid(W, bits)
+    _, perm = oracle.sensitivity_order(W, diag, sc, zp, bits)
+    ref = oracle.quantize_layer(W, Hinv, perm, sc, zp, bits, H_undamped=H, want_prer=True)
+    codes, What, loss = _sweep(W, Hinv, perm, sc, zp, bits, H)
+    nm = compare_codes(codes, ref)
+    assert nm == 0
+    assert np.array_equal(What, ref["What"])
+    assert abs(loss - ref["loss"]) <= 1e-9 * ref["loss"]
+
+
+def test_identity_inverse_hessian_gives_round_to_nearest():
+    W, _ = _layer(40, 130, 8, 600)
+    W[0, :8] = 0.0
+    for bits in (2, 4, 8):
+        sc, zp = oracle.minmax_grid(W, bits)
+        perm = np.random.Generator(np.random.PCG64(1)).permutation(130).astype(np.int32)
+        codes, What, _ = _sweep(W, np.eye(130), perm, sc, zp, bits)
+        v = np.clip(np.rint(W.astype(np.float64) / sc[:, None].astype(np.float64)) + zp[:, None], 0, 2 ** bits - 1)
+        assert np.array_equal(codes, v.astype(np.uint8))
+        assert np.array_equal(What, (sc[:, None].astype(np.float64) * (v - zp[:, None])).astype(np.float32))
+
+
+def test_invalid_permutation_is_reported_not_followed():
+    W, X = _layer(8, 64, 100, 601)
+    Hinv, diag, _ = oracle.prepare_hinv(oracle.hessian_accumulate(X))
+    sc, zp = oracle.minmax_grid(W, 4)
+    perm = np.arange(64, dtype=np.int32)
+    perm[10] = 3                     # repeated entry
+    perm[20] = 9999                  # out of range
+    codes = torch.empty((8, 64), dtype=torch.uint8, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.quantize_layer(_cuda(W), _cuda(Hinv), _cuda(perm), _cuda(sc), _cuda(zp), 4, codes, None, None, None, ws, st)
+    torch.cuda.synchronize()
+    with pytest.raises(ptq.PtqError) as ei:
+        ptq.check_status(st)
+    assert ei.value.code == ptq.ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------------------------------ whole path
+@pytest.mark.parametrize("rows,cols,n,bits,xdist", [
+    (64, 128, 1024, 4, "halfnormal"),
+    (37, 147, 260, 4, "halfnormal"),          # ragged: 7x7 stem width, n not a multiple of the K block
+    (255, 128, 512, 8, "silu"),               # YOLO head: 255 rows
+    (32, 108, 256, 4, "silu"),                # 6x6 stem
+    (100, 300, 200, 3, "normal"),             # cols > n: rank-deficient before damping
+    (1, 1, 4, 4, "normal"),                   # degenerate 1x1 layer
+    (3, 2, 1, 2, "halfnormal"),
+])
+def test_whole_path_matches_oracle(rows, cols, n, bits, xdist):
+    W, X = _layer(rows, cols, n, 700 + rows + cols, bits, xdist)
+    ref = oracle_layer(W, X, bits)
+    g = gpu_layer(W, X, bits)
+    assert np.max(np.abs(g["H"] - ref["H"])) <= 2e-12 * np.max(np.abs(ref["H"]))
+    assert assert_layer_parity(g, ref) == 0
+
+
+def test_config1_bit_exact_and_deterministic():
+    spec = wl.config1()[0]
+    W, X = wl.make_layer(spec)
+    ref = oracle_layer(W, X, spec.bits, spec.damp)
+    runs = [gpu_layer(W, X, spec.bits, spec.damp) for _ in range(3)]
+    assert assert_layer_parity(runs[0], ref) == 0
+    for r in runs[1:]:
+        for k in ("H", "Hinv", "S", "perm", "codes", "What", "loss"):
+            assert np.array_equal(r[k], runs[0][k]), f"{k} is not bit-identical across runs"
+
+
+@pytest.mark.parametrize("mode", [ptq.SCORE_PRUNE, ptq.SCORE_ERR, ptq.SCORE_W, ptq.SCORE_NONE])
+def test_ordering_modes_whole_path(mode):
+    W, X = _layer(48, 160, 400, 800 + mode)
+    ref = oracle_layer(W, X, 4, score_mode=mode)
+    g = gpu_layer(W, X, 4, score_mode=mode)
+    assert assert_layer_parity(g, ref) == 0
+
+
+def test_absolute_damping_whole_path():
+    W, X = _layer(24, 96, 300, 810)
+    ref = oracle_layer(W, X, 4, damp=0.1, damp_mode=oracle.DAMP_ABS)
+    g = gpu_layer(W, X, 4, damp=0.1, damp_mode=ptq.DAMP_ABS)
+    assert assert_layer_parity(g, ref) == 0
+
+
+def test_config2_full_size():
+    """The bench workload (256 x 2304, N = 4096, 30 % zeros) at full size, in the bench's launch configuration."""
+    spec = wl.config2()[0]
+    W, X = wl.make_layer(spec)
+    ref = oracle_layer(W, X, spec.bits, spec.damp)
+    g = gpu_layer(W, X, spec.bits, spec.damp)
+    assert np.max(np.abs(g["H"] - ref["H"])) <= 2e-12 * np.max(np.abs(ref["H"]))
+    assert np.max(np.abs(g["Hinv"] - ref["Hinv"])) <= 1e-10 * np.max(np.abs(ref["Hinv"]))
+    assert_layer_parity(g, ref)
+    assert abs(float(g["loss"][0]) - oracle.loss_direct(W, g["What"], X)) <= 1e-9 * ref["loss"]
