@@ -1,0 +1,347 @@
+#!/usr/bin/env python
+"""Benchmark of the per-layer quantizer hot path on B200.
+
+One "step" = one pass of the whole hot path over one synthetic layer: Hessian H = 2 X X^T, damped
+inverse, grid, column scores + order, column-synchronous quantization sweep, codes / What / loss.
+Workload at N = 1: the ResNet-50-shaped 3x3 convolution as a matrix (W 256 x 2304, X 2304 x 4096 with
+30 % exact zeros, 4-bit per-row asymmetric grid, damping 0.01 * mean(diag H)).
+
+`python bench.py [--gpus N] [--steps K] [--warmup W]` prints ONE JSON line (rank 0).  With N > 1 (torchrun)
+every rank quantizes its own replica of the layer (the path is single-GPU: no collective on the data path);
+`value` is the weights quantized per second by all ranks together, timed on the device, max over ranks.
+`--impl reference` times the float64 CPU oracle on the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2509_05576_b200 import workloads as wl  # noqa: E402
+
+METRIC = "weights quantized per second, whole per-layer path (ms_per_step = layer quantize time)"
+UNIT = "weights/s"
+FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12      # 148 SMs x 64 FP64 FMA / clk x 1965 MHz = 37.2
+INT8_OVER_BF16 = 2.0                                   # nominal dense 4.5 / 2.25 PFLOP/s
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"], "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = str(gpu_index)
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu, f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def bench_spec(rank=0):
+    spec = wl.config2()[0]
+    if rank:
+        spec = wl.LayerSpec(spec.name, spec.rows, spec.cols, spec.n, spec.bits, spec.w_dist, spec.x_dist,
+                            spec.seed + 100 * rank, spec.damp)
+    return spec
+
+
+def workload_config(spec, n_gpus):
+    return {"workload": f"ResNet-50-shaped 3x3 conv as matrix: W {spec.rows}x{spec.cols} Kaiming-normal fp32, "
+                        f"X {spec.cols}x{spec.n} half-normal with 30% exact zeros, {spec.bits}-bit per-row asymmetric "
+                        f"min-max grid, damping {spec.damp}*mean(diag H), seed {spec.seed}",
+            "rows": spec.rows, "cols": spec.cols, "n": spec.n, "bits": spec.bits,
+            "l2": "L2 flushed (256 MiB write) before every timed step",
+            "parallelism": "single GPU" if n_gpus == 1 else f"{n_gpus} independent replicas, one layer per GPU"}
+
+
+# ------------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle as it stands
+# ------------------------------------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    spec = bench_spec()
+    W, X = wl.make_layer(spec)
+    cores = oracle.num_threads()
+    for _ in range(args.warmup):
+        oracle.run_layer(W, X, spec.bits, spec.damp)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.run_layer(W, X, spec.bits, spec.damp)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = spec.weights / dt
+    sample = f"the whole {spec.rows}x{spec.cols} layer (N={spec.n}) per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": workload_config(spec, 1),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+    return 0
+
+
+# ------------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------------
+def algorithmic_work(spec):
+    """Algorithmic flops of one step per kernel (MAC = 2 flops), used for the roofline of the dominant kernel."""
+    r, c, n = spec.rows, spec.cols, spec.n
+    return {
+        "gram_i8_tcgen05": ("tensor", c * (c + 1) * n),            # symmetric half of 2 X X^T
+        "dgemm_chol_trailing": ("alu", 2 * (c ** 3 / 3.0)),         # two Cholesky factorisations, c^3/3 flops each
+        "dgemm_trtri": ("alu", c ** 3 / 3.0),
+        "dgemm_lauum": ("alu", c ** 3 / 3.0),
+        "dgemm_w_update": ("alu", float(r) * c * c),                # r c^2 / 2 MACs
+        "dgemm_loss": ("alu", 2.0 * r * c * c),
+        "potrf_diag": ("alu", 2 * (c / 64.0) * (64 ** 3 / 3.0)),
+        "panel_solve": ("alu", 2 * (c * c / 2.0) * 64),
+        "colloop_block": ("alu", float(r) * c * 64),
+    }
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_05576_b200 import ptq
+    import oracle
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the quantizer has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ptq.lib()
+
+    spec = bench_spec(rank)
+    W, X = wl.make_layer(spec)
+    Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
+    bufs = ptq.LayerBuffers(spec.rows, spec.cols)
+    ws = ptq.Workspace()
+    stream = torch.cuda.current_stream()
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step(events=None):
+        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, bufs=bufs, ws=ws, stream=stream, events=events)
+
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    ptq.check_status(bufs.status, "warm-up")
+
+    # ---- timed region: K steps, device time by CUDA events on the launching stream, L2 flushed between steps
+    sampler = ClockSampler(os.environ.get("CUDA_VISIBLE_DEVICES", str(local)).split(",")[0] if world == 1 else local)
+    starts = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    ends = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    launches0 = ptq.launch_count()
+    barrier()
+    sampler.start()
+    for k in range(args.steps):
+        flush.fill_(k & 0xFF)
+        starts[k].record(stream)
+        step()
+        ends[k].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    launches = ptq.launch_count() - launches0
+    ptq.check_status(bufs.status, "timed region")
+    total_ms = sum(a.elapsed_time(b) for a, b in zip(starts, ends))
+    t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * spec.weights / (ms_per_step * 1e-3)
+
+    # ---- per-stage times (events around each C-ABI call) and per-kernel times (library launch profiler)
+    stage_ms = {}
+    for _ in range(3):
+        ev = []
+        flush.fill_(3)
+        step(ev)
+        torch.cuda.synchronize()
+        for name, a, b in ev:
+            stage_ms.setdefault(name, []).append(a.elapsed_time(b))
+    stage_ms = {k: float(np.median(v)) for k, v in stage_ms.items()}
+    ptq.profile_enable(True)
+    prof_steps = 3
+    for _ in range(prof_steps):
+        flush.fill_(5)
+        step()
+    torch.cuda.synchronize()
+    prof = ptq.profile_read()
+    ptq.profile_enable(False)
+    kernels = {k: {"ms_per_step": ms / prof_steps, "launches_per_step": cnt // prof_steps} for k, (ms, cnt) in prof.items()}
+    dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    peaks = load_peaks()
+    work = algorithmic_work(spec)
+    bound, flops = work.get(dominant, ("alu", 0.0))
+    dom = kernels[dominant]
+    per_launch_ms = dom["ms_per_step"] / max(dom["launches_per_step"], 1)
+    achieved = flops / max(dom["launches_per_step"], 1) / (per_launch_ms * 1e-3) / 1e12
+    if bound == "tensor":
+        peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+        peak_note = f"int8 dense = {peaks['source']} bf16 burst {peaks['bf16_tflops']} TF/s x nominal ratio 2"
+    else:
+        peak = FP64_PEAK_TFLOPS
+        peak_note = "float64 FMA pipe: 148 SMs x 64 FMA/clk x 2 x 1965 MHz"
+    traffic = None
+    tpath = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if os.path.exists(tpath):
+        with open(tpath) as f:
+            traffic = json.load(f).get(dominant)
+    roofline = {"kernel": dominant, "bound": bound, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": traffic, "peak_source": peak_note,
+                "launch_ms": per_launch_ms, "launches_per_step": dom["launches_per_step"],
+                "algorithmic_flops_per_step": flops}
+    gram = kernels.get("gram_i8_tcgen05")
+    if gram:
+        gflops = work["gram_i8_tcgen05"][1]
+        gach = gflops / (gram["ms_per_step"] * 1e-3) / 1e12
+        roofline["gram_i8_tcgen05"] = {"bound": "tensor", "achieved": gach, "issued": gach * 21,
+                                       "peak": peaks["bf16_tflops"] * INT8_OVER_BF16, "unit": "TFLOP/s",
+                                       "frac": gach / (peaks["bf16_tflops"] * INT8_OVER_BF16),
+                                       "frac_issued": gach * 21 / (peaks["bf16_tflops"] * INT8_OVER_BF16)}
+
+    # ---- end to end through the C-ABI with HOST buffers: H2D of W and X, the path, D2H of codes and loss
+    Wh, Xh = torch.from_numpy(W).pin_memory(), torch.from_numpy(X).pin_memory()
+    codes_h = torch.empty((spec.rows, spec.cols), dtype=torch.uint8).pin_memory()
+    loss_h = torch.empty(1, dtype=torch.float64).pin_memory()
+    Wdev, Xdev = torch.empty_like(Wd), torch.empty_like(Xd)
+
+    def e2e_step():
+        Wdev.copy_(Wh, non_blocking=True)
+        Xdev.copy_(Xh, non_blocking=True)
+        ptq.quantize_layer_full(Wdev, Xdev, spec.bits, spec.damp, bufs=bufs, ws=ws, stream=stream)
+        codes_h.copy_(bufs.codes, non_blocking=True)
+        loss_h.copy_(bufs.loss, non_blocking=True)
+
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e2e_steps = max(3, min(args.steps, 10))
+    e2e_ms = 0.0
+    for k in range(e2e_steps):
+        flush.fill_(k & 0xFF)
+        e0.record(stream)
+        e2e_step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        e2e_ms += e0.elapsed_time(e1)
+    barrier()
+    t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * spec.weights / (float(t.item()) / e2e_steps * 1e-3)
+    e2e = {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(W.nbytes + X.nbytes),
+           "d2h_bytes_per_step": int(codes_h.numel() + 8), "ms_per_step": float(t.item()) / e2e_steps}
+
+    # ---- CPU baseline: the oracle as it stands, rank 0 at N = 1 only
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        t0 = time.perf_counter()
+        ref = oracle.run_layer(W, X, spec.bits, spec.damp)
+        dt = time.perf_counter() - t0
+        cpu_baseline = {"value": spec.weights / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                        "sample": f"the whole {spec.rows}x{spec.cols} layer (N={spec.n}), one pass, {dt:.2f} s",
+                        "codes_equal_to_gpu": bool(np.array_equal(ref["codes"], bufs.codes.cpu().numpy())),
+                        "order_equal_to_gpu": bool(np.array_equal(ref["perm"], bufs.perm.cpu().numpy()))}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64 (Gram: exact int8 slices on tcgen05, int32 accumulate)",
+            "data": "synthetic", "config": workload_config(spec, world), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "stages_ms": stage_ms, "kernels": kernels,
+            "context": "paper: ResNet-50 whole-model 80 s (FastOBQ) vs 9287 s (OBQ), hardware not stated"}))
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

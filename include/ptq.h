@@ -128,6 +128,22 @@ int ptq_quantize_layer(const float *W, int rows, int cols, int64_t ldw, const do
 const char *ptq_status_string(int code);
 int ptq_version(void);
 
+/*
+ * Launch accounting (instrumentation; the paper has no counterpart).  Host-side state of the calling process.
+ *   ptq_kernel_count / ptq_kernel_name : the library's kernels, by id.
+ *   ptq_launch_count(id)   : launches of kernel `id` since the library was loaded; id < 0 gives the total.
+ *   ptq_profile_enable(on) : while on, every launch is bracketed by CUDA events on its stream (this perturbs
+ *                            timing, so profile on passes that are not themselves being timed); each call clears
+ *                            the records taken so far.
+ *   ptq_profile_read(id, total_ms, launches) : host pointers; waits for the recorded events and sums the device
+ *                            time of kernel `id` over the recorded launches.
+ */
+int ptq_kernel_count(void);
+const char *ptq_kernel_name(int kernel_id);
+long long ptq_launch_count(int kernel_id);
+int ptq_profile_enable(int on);
+int ptq_profile_read(int kernel_id, double *total_ms, long long *launches);
+
 #ifdef __cplusplus
 }
 #endif

@@ -30,6 +30,43 @@ extern "C" {
 
 int ptq_version(void) { return 1; }
 
+int ptq_kernel_count(void) { return K_COUNT; }
+
+const char* ptq_kernel_name(int kernel_id) { return kernel_name(kernel_id); }
+
+long long ptq_launch_count(int kernel_id) {
+    const Profiler& p = profiler();
+    if (kernel_id >= 0 && kernel_id < K_COUNT) return p.launches[kernel_id];
+    long long total = 0;
+    for (int k = 0; k < K_COUNT; ++k) total += p.launches[k];
+    return total;
+}
+
+int ptq_profile_enable(int on) {
+    Profiler& p = profiler();
+    p.clear();
+    p.on = on != 0;
+    return PTQ_OK;
+}
+
+int ptq_profile_read(int kernel_id, double* total_ms, long long* launches) {
+    Profiler& p = profiler();
+    if (kernel_id < 0 || kernel_id >= K_COUNT || !total_ms || !launches) return PTQ_ERR_INVALID_ARG;
+    double ms = 0.0;
+    long long cnt = 0;
+    for (const auto& r : p.recs) {
+        if (r.id != kernel_id) continue;
+        if (cudaEventSynchronize(r.b) != cudaSuccess) return PTQ_ERR_CUDA;
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, r.a, r.b) != cudaSuccess) return PTQ_ERR_CUDA;
+        ms += (double)t;
+        ++cnt;
+    }
+    *total_ms = ms;
+    *launches = cnt;
+    return PTQ_OK;
+}
+
 const char* ptq_status_string(int code) {
     switch (code) {
         case PTQ_OK: return "ok";
@@ -91,14 +128,14 @@ int ptq_hessian_accumulate_f64(double* H, const float* X, int cols, int n, int64
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE_F64, 0, cols, n)) return PTQ_ERR_WORKSPACE;
     Carver cv(ws);
     double* Xd = cv.take<double>((size_t)cols * n);
-    convert_f32_f64_kernel<<<dim3(grid_x_for(n, 256), cols), 256, 0, stream>>>(X, cols, n, ldx, Xd);
+    { Launch l(K_CONVERT_F64, stream); convert_f32_f64_kernel<<<dim3(grid_x_for(n, 256), cols), 256, 0, stream>>>(X, cols, n, ldx, Xd); }
     GemmParams g = gemm_defaults();
     g.A = Xd; g.lda = n; g.a_trans = 0;
     g.B = Xd; g.ldb = n; g.b_trans = 1;
     g.C = H; g.ldc = cols;
     g.M = cols; g.N = cols; g.K = n;
     g.alpha = 2.0; g.beta = 1.0; g.upper_only = 1; g.mirror = 1;
-    return launch_dgemm(g, 1, stream);
+    return launch_dgemm(K_DGEMM_GRAM, g, 1, stream);
 }
 
 int ptq_hessian_accumulate(double* H, const float* X, int cols, int n, int64_t ldx, void* ws, size_t ws_bytes,
@@ -121,8 +158,8 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     Carver cv(ws);
     double* R = cv.take<double>((size_t)n * n);
     double* V = cv.take<double>((size_t)n * n);
-    lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status);
-    damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out);
+    { Launch l(K_LAMBDA, stream); lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status); }
+    { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out); }
     int st = cholesky_upper(R, n, status, stream);
     if (st) return st;
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
@@ -130,7 +167,7 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     if (st) return st;
     st = lauum_upper(V, Hinv, n, stream);
     if (st) return st;
-    extract_diag_kernel<<<cdiv(n, 256), 256, 0, stream>>>(Hinv, n, Hinv_diag);
+    { Launch l(K_EXTRACT_DIAG, stream); extract_diag_kernel<<<cdiv(n, 256), 256, 0, stream>>>(Hinv, n, Hinv_diag); }
     return launch_status();
 }
 
@@ -139,7 +176,7 @@ int ptq_minmax_grid(const float* W, int rows, int cols, int64_t ldw, int bits, f
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!W || !scale || !zero || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8)
         return PTQ_ERR_INVALID_ARG;
-    minmax_grid_kernel<<<rows, 256, 0, stream>>>(W, rows, cols, ldw, bits, scale, zero, status);
+    { Launch l(K_MINMAX_GRID, stream); minmax_grid_kernel<<<rows, 256, 0, stream>>>(W, rows, cols, ldw, bits, scale, zero, status); }
     return launch_status();
 }
 
@@ -156,11 +193,13 @@ int ptq_sensitivity_order(const float* W, int rows, int cols, int64_t ldw, const
     Carver cv(ws);
     const int chunks = cdiv(rows, kScoreRowChunk);
     double* partial = cv.take<double>((size_t)chunks * cols);
-    if (score_mode != PTQ_SCORE_NONE)
+    if (score_mode != PTQ_SCORE_NONE) {
+        Launch l(K_SCORE_PARTIAL, stream);
         score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
                                                                               score_mode, partial);
-    score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status);
-    rank_sort_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(S, cols, perm);
+    }
+    { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status); }
+    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(S, cols, perm); }
     return launch_status();
 }
 
@@ -193,17 +232,20 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
         cudaSuccess)
         return PTQ_ERR_CUDA;
-    perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status);
-    gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U);
-    gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp);
+    { Launch l(K_PERM_CHECK, stream); perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status); }
+    { Launch l(K_GATHER_SYM, stream); gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U); }
+    { Launch l(K_GATHER_W, stream); gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp); }
     int st = cholesky_upper(U, n, status, stream);   // blocked Eq. 12
     if (st) return st;
 
     const int row_ctas = cdiv(rows, kRowsPerCta);
     for (int p0 = 0; p0 < n; p0 += kNB) {
         const int kb = n - p0 < kNB ? n - p0 : kNB;
-        colloop_block_kernel<<<row_ctas, 128, kColloopSmem, stream>>>(Wp, rows, n, p0, kb, U, scale, zero, bits, E,
-                                                                      codes_p);
+        {
+            Launch l(K_COLLOOP_BLOCK, stream);
+            colloop_block_kernel<<<row_ctas, 128, kColloopSmem, stream>>>(Wp, rows, n, p0, kb, U, scale, zero, bits, E,
+                                                                          codes_p);
+        }
         const int rest = n - p0 - kb;
         if (rest <= 0) break;
         GemmParams g = gemm_defaults();     // deferred Eq. 11: W[:, later] -= E[:, block] U[block, later]
@@ -212,14 +254,17 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
         g.C = Wp + p0 + kb; g.ldc = n;
         g.M = rows; g.N = rest; g.K = kb;
         g.alpha = -1.0; g.beta = 1.0;
-        st = launch_dgemm(g, 1, stream);
+        st = launch_dgemm(K_DGEMM_WUPDATE, g, 1, stream);
         if (st) return st;
     }
 
     const bool want_loss = H_undamped && loss_out;
     double* dW = want_loss ? Wp : nullptr;
-    finalize_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(codes_p, invperm, W, rows, n, ldw, scale, zero,
-                                                                       codes, What, dW);
+    {
+        Launch l(K_FINALIZE, stream);
+        finalize_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(codes_p, invperm, W, rows, n, ldw, scale,
+                                                                           zero, codes, What, dW);
+    }
     if (want_loss) {
         GemmParams g = gemm_defaults();     // sum_ij (dW H)_ij dW_ij
         g.A = dW; g.lda = n; g.a_trans = 0;
@@ -227,9 +272,9 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
         g.M = rows; g.N = n; g.K = n;
         g.D = dW; g.ldd = n; g.partials = partials;
         dim3 grid;
-        st = launch_dgemm(g, 1, stream, 64, &grid);
+        st = launch_dgemm(K_DGEMM_LOSS, g, 1, stream, 64, &grid);
         if (st) return st;
-        sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y), 0.5, loss_out);
+        { Launch l(K_SUM_PARTIALS, stream); sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y), 0.5, loss_out); }
     }
     return launch_status();
 }

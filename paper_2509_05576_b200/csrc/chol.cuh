@@ -102,17 +102,17 @@ __global__ void __launch_bounds__(128) panel_solve_kernel(double* __restrict__ A
 inline int cholesky_upper(double* A, int n, int32_t* status, cudaStream_t stream) {
     for (int k0 = 0; k0 < n; k0 += kNB) {
         const int kb = n - k0 < kNB ? n - k0 : kNB;
-        potrf_diag_kernel<<<1, 256, 0, stream>>>(A, n, k0, kb, status);
+        { Launch l(K_POTRF_DIAG, stream); potrf_diag_kernel<<<1, 256, 0, stream>>>(A, n, k0, kb, status); }
         const int rest = n - k0 - kb;
         if (rest <= 0) break;
-        panel_solve_kernel<<<cdiv(rest, 128), 128, 0, stream>>>(A, n, k0, kb, n);
+        { Launch l(K_PANEL_SOLVE, stream); panel_solve_kernel<<<cdiv(rest, 128), 128, 0, stream>>>(A, n, k0, kb, n); }
         GemmParams g = gemm_defaults();     // A22 -= U12^T U12 on the upper tiles
         g.A = A + (int64_t)k0 * n + k0 + kb; g.lda = n; g.a_trans = 1;
         g.B = g.A; g.ldb = n; g.b_trans = 0;
         g.C = A + (int64_t)(k0 + kb) * n + k0 + kb; g.ldc = n;
         g.M = rest; g.N = rest; g.K = kb;
         g.alpha = -1.0; g.beta = 1.0; g.upper_only = 1;
-        int st = launch_dgemm(g, 1, stream);
+        int st = launch_dgemm(K_DGEMM_CHOL, g, 1, stream);
         if (st) return st;
     }
     return launch_status();
@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(kNB) diag_inverse_kernel(const double* __restr
 // V = R^-1 for upper-triangular R (n x n).  V must be zero on entry; T is n x n scratch.
 // Recursive halving: with R = [R11 R12; 0 R22], V12 = -V11 (R12 V22); all pairs of one level run as one batch.
 inline int trtri_upper(const double* R, double* V, double* T, int n, cudaStream_t stream) {
-    diag_inverse_kernel<<<cdiv(n, kNB), kNB, 0, stream>>>(R, V, n, n);
+    { Launch l(K_DIAG_INVERSE, stream); diag_inverse_kernel<<<cdiv(n, kNB), kNB, 0, stream>>>(R, V, n, n); }
     for (int64_t s = kNB; s < n; s *= 2) {
         const int pairs = (int)((n + 2 * s - 1) / (2 * s));
         const int64_t step = 2 * s * ((int64_t)n + 1);
@@ -161,7 +161,7 @@ inline int trtri_upper(const double* R, double* V, double* T, int n, cudaStream_
         g.M = (int)s; g.N = (int)s; g.K = (int)s;
         g.ragN_lim = n - (int)s; g.ragN_step = (int)(2 * s); g.k_is_n = 1;
         g.kend_mode = 1;
-        int st = launch_dgemm(g, pairs, stream);
+        int st = launch_dgemm(K_DGEMM_TRTRI, g, pairs, stream);
         if (st) return st;
         GemmParams h = gemm_defaults();     // V12 = -V11 T12   (V11 upper: k starts at the tile's first row)
         h.A = V; h.lda = n; h.a_trans = 0; h.batch_a = step;
@@ -171,7 +171,7 @@ inline int trtri_upper(const double* R, double* V, double* T, int n, cudaStream_
         h.ragN_lim = n - (int)s; h.ragN_step = (int)(2 * s);
         h.kbeg_mode = 2;
         h.alpha = -1.0;
-        st = launch_dgemm(h, pairs, stream);
+        st = launch_dgemm(K_DGEMM_TRTRI, h, pairs, stream);
         if (st) return st;
     }
     return launch_status();
@@ -185,7 +185,7 @@ inline int lauum_upper(const double* V, double* Hinv, int n, cudaStream_t stream
     g.C = Hinv; g.ldc = n;
     g.M = n; g.N = n; g.K = n;
     g.kbeg_mode = 1; g.upper_only = 1; g.mirror = 1;
-    return launch_dgemm(g, 1, stream);
+    return launch_dgemm(K_DGEMM_LAUUM, g, 1, stream);
 }
 
 __global__ void extract_diag_kernel(const double* __restrict__ A, int n, double* __restrict__ d) {

@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <vector>
 
 #include "../../include/ptq.h"
 
@@ -38,5 +39,58 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 inline int launch_status() { return cudaGetLastError() == cudaSuccess ? PTQ_OK : PTQ_ERR_CUDA; }
 
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// ---------------------------------------------------------------------------------------------------------
+// Launch accounting.  Every kernel launch of the library goes through a Launch scope: it always counts the
+// launch, and, while profiling is enabled, brackets it with CUDA events on the launching stream so that the
+// bench can read per-kernel device time live.  Profiling adds event records between kernels, so it is used on
+// separate, untimed passes.
+// ---------------------------------------------------------------------------------------------------------
+enum KernelId {
+    K_GRAM_SPLIT = 0, K_GRAM_I8, K_CONVERT_F64, K_DGEMM_GRAM, K_LAMBDA, K_DAMP_COPY, K_POTRF_DIAG, K_PANEL_SOLVE,
+    K_DGEMM_CHOL, K_DIAG_INVERSE, K_DGEMM_TRTRI, K_DGEMM_LAUUM, K_EXTRACT_DIAG, K_MINMAX_GRID, K_SCORE_PARTIAL,
+    K_SCORE_FINAL, K_RANK_SORT, K_PERM_CHECK, K_GATHER_SYM, K_GATHER_W, K_COLLOOP_BLOCK, K_DGEMM_WUPDATE, K_FINALIZE,
+    K_DGEMM_LOSS, K_SUM_PARTIALS, K_COUNT
+};
+
+inline const char* kernel_name(int id) {
+    static const char* names[K_COUNT] = {
+        "gram_split", "gram_i8_tcgen05", "convert_f64", "dgemm_gram_f64", "lambda", "damp_copy", "potrf_diag",
+        "panel_solve", "dgemm_chol_trailing", "diag_inverse", "dgemm_trtri", "dgemm_lauum", "extract_diag",
+        "minmax_grid", "score_partial", "score_final", "rank_sort", "perm_check", "gather_sym", "gather_w",
+        "colloop_block", "dgemm_w_update", "finalize", "dgemm_loss", "sum_partials"};
+    return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
+}
+
+struct Profiler {
+    bool on = false;
+    long long launches[K_COUNT] = {};
+    struct Rec { int id; cudaEvent_t a, b; };
+    std::vector<Rec> recs;
+    std::vector<cudaEvent_t> pool;
+    cudaEvent_t get() {
+        if (!pool.empty()) { cudaEvent_t e = pool.back(); pool.pop_back(); return e; }
+        cudaEvent_t e = nullptr;
+        cudaEventCreate(&e);
+        return e;
+    }
+    void clear() {
+        for (auto& r : recs) { pool.push_back(r.a); pool.push_back(r.b); }
+        recs.clear();
+    }
+};
+inline Profiler& profiler() { static Profiler p; return p; }
+
+struct Launch {
+    int id; cudaStream_t s; cudaEvent_t a = nullptr, b = nullptr;
+    Launch(int id_, cudaStream_t s_) : id(id_), s(s_) {
+        Profiler& p = profiler();
+        ++p.launches[id];
+        if (p.on) { a = p.get(); b = p.get(); if (a) cudaEventRecord(a, s); }
+    }
+    ~Launch() {
+        if (a && b) { cudaEventRecord(b, s); profiler().recs.push_back({id, a, b}); }
+    }
+};
 
 }  // namespace ptq

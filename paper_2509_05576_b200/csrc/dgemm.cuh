@@ -204,7 +204,7 @@ inline GemmParams gemm_defaults() {
 }
 
 // Launches with 128x128 tiles when that still fills the GPU, else 64x64.  Also reports the grid used.
-inline int launch_dgemm(const GemmParams& p, int batches, cudaStream_t stream, int force_bt = 0,
+inline int launch_dgemm(int kernel_id, const GemmParams& p, int batches, cudaStream_t stream, int force_bt = 0,
                         dim3* grid_out = nullptr) {
     static bool attr_done = false;
     if (!attr_done) {
@@ -222,6 +222,7 @@ inline int launch_dgemm(const GemmParams& p, int batches, cudaStream_t stream, i
     }
     dim3 grid(cdiv(p.N, bt), cdiv(p.M, bt), batches);
     if (grid_out) *grid_out = grid;
+    Launch scope(kernel_id, stream);
     if (bt == 128)
         dgemm_kernel<128><<<grid, kGemmThreads, gemm_smem_bytes<128>(), stream>>>(p);
     else

@@ -450,16 +450,22 @@ inline int gram_accumulate(double* H, const float* X, int cols, int n, int64_t l
         const int nc = n - c0 < kGramMaxChunk ? n - c0 : kGramMaxChunk;
         const int n_pad = cdiv(nc, 128) * 128;
         const int vec_ok = (aligned16(X) && (ldx & 3) == 0) ? 1 : 0;
-        gram_split_kernel<<<cols_pad, 256, 0, stream>>>(X + c0, cols, nc, ldx, cols_pad, n_pad, vec_ok, Q, shifts,
-                                                        status);
+        {
+            Launch l(K_GRAM_SPLIT, stream);
+            gram_split_kernel<<<cols_pad, 256, 0, stream>>>(X + c0, cols, nc, ldx, cols_pad, n_pad, vec_ok, Q, shifts,
+                                                            status);
+        }
         CUtensorMap mapA, mapB;
         int st = make_slice_map(&mapA, Q, cols_pad, n_pad, kGramTM);
         if (st) return st;
         st = make_slice_map(&mapB, Q, cols_pad, n_pad, kGramTN);
         if (st) return st;
         const int grid = num_tiles < num_sms ? num_tiles : num_sms;
-        gram_i8_kernel<<<grid, kGramThreads, kGramSmemBytes, stream>>>(mapA, mapB, H, cols, n_pad, shifts, num_tiles,
-                                                                     nbj, status);
+        {
+            Launch l(K_GRAM_I8, stream);
+            gram_i8_kernel<<<grid, kGramThreads, kGramSmemBytes, stream>>>(mapA, mapB, H, cols, n_pad, shifts,
+                                                                         num_tiles, nbj, status);
+        }
         if (cudaGetLastError() != cudaSuccess) return PTQ_ERR_CUDA;
     }
     return PTQ_OK;

@@ -21,7 +21,8 @@ SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
 CALL_HESSIAN_ACCUMULATE, CALL_PREPARE_HINV, CALL_SENSITIVITY_ORDER, CALL_QUANTIZE_LAYER, CALL_HESSIAN_ACCUMULATE_F64 = range(5)
 
 EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
-           "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_quantize_layer", "ptq_status_string", "ptq_version"]
+           "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
+           "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
 
 
 class PtqError(RuntimeError):
@@ -59,12 +60,39 @@ def lib():
         L.ptq_status_string.argtypes = [c_int]
         L.ptq_status_string.restype = ctypes.c_char_p
         L.ptq_version.restype = c_int
+        L.ptq_kernel_count.restype = c_int
+        L.ptq_kernel_name.argtypes = [c_int]
+        L.ptq_kernel_name.restype = ctypes.c_char_p
+        L.ptq_launch_count.argtypes = [c_int]
+        L.ptq_launch_count.restype = ctypes.c_longlong
+        L.ptq_profile_enable.argtypes = [c_int]
+        L.ptq_profile_read.argtypes = [c_int, ctypes.POINTER(c_double), ctypes.POINTER(ctypes.c_longlong)]
         _lib = L
     return _lib
 
 
 def status_string(code: int) -> str:
     return lib().ptq_status_string(int(code)).decode()
+
+
+def launch_count(kernel_id: int = -1) -> int:
+    """Kernel launches made by the library in this process (all kernels when kernel_id < 0)."""
+    return int(lib().ptq_launch_count(int(kernel_id)))
+
+
+def profile_enable(on: bool):
+    _check(lib().ptq_profile_enable(1 if on else 0), "ptq_profile_enable")
+
+
+def profile_read():
+    """Per-kernel device time of the launches recorded since ``profile_enable(True)``: {name: (ms, launches)}."""
+    out = {}
+    for k in range(lib().ptq_kernel_count()):
+        ms, cnt = c_double(0.0), ctypes.c_longlong(0)
+        _check(lib().ptq_profile_read(k, ctypes.byref(ms), ctypes.byref(cnt)), "ptq_profile_read")
+        if cnt.value:
+            out[lib().ptq_kernel_name(k).decode()] = (ms.value, cnt.value)
+    return out
 
 
 def workspace_bytes(call_id: int, rows: int, cols: int, n: int) -> int:
