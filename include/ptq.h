@@ -38,7 +38,8 @@ typedef enum {
     PTQ_ERR_NONFINITE = 5,
     PTQ_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired */
     PTQ_ERR_CUDA = 7,        /* a CUDA runtime call failed on the host */
-    PTQ_ERR_UNSUPPORTED = 8
+    PTQ_ERR_UNSUPPORTED = 8,
+    PTQ_ERR_STATIC_SCRATCH = 9 /* ptq_sensitivity_order_static: rows x cols beyond the built-in scratch array */
 } ptq_status;
 
 /* Damping (Implementation Details: a constant is added to the diagonal of H). */
@@ -108,6 +109,33 @@ int ptq_minmax_grid(const float *W, int rows, int cols, int64_t ldw, int bits, f
 int ptq_sensitivity_order(const float *W, int rows, int cols, int64_t ldw, const double *Hinv_diag, const float *scale,
                           const float *zero, int bits, int score_mode, double *S, int32_t *perm, void *ws,
                           size_t ws_bytes, int32_t *status, void *stream);
+
+/*
+ * ptq_sensitivity_order for callers that cannot hand the library any scratch memory.  (The paper has no
+ * counterpart: this is a packaging variant of the call above, with the same inputs, outputs and arithmetic.)
+ *
+ * Who needs it: code that runs where device allocation is off limits -- inside a region that must not call
+ * cudaMalloc (a latency-critical serving loop, a process whose memory pool is owned and fully handed out by
+ * another component, a plug-in that is given device pointers but no allocator) -- and that therefore cannot size
+ * and provide the `ws` buffer the ordinary call asks for.  This entry point takes no workspace: the per-row-chunk
+ * partial sums live in an array compiled into the library, PTQ_STATIC_SCRATCH_BYTES large.  Every device that loads
+ * the library carries that array until the process exits, whether or not this function is ever called.
+ *
+ * Limits and rules
+ *   - ceil(rows / 64) * cols * 8 bytes must not exceed PTQ_STATIC_SCRATCH_BYTES (e.g. 4096 x 11008 fits);
+ *     larger problems return PTQ_ERR_STATIC_SCRATCH and launch nothing.
+ *   - It never calls cudaMalloc, cudaFree or any allocating routine.  The first call on each device looks up the
+ *     array's device address (cudaGetSymbolAddress, with the caller's device current) and keeps it; make that
+ *     first call outside any stream capture.
+ *   - All calls on one device share the one array, and it keeps whatever the previous call left there.  The
+ *     kernels overwrite every element they later read, so no clearing is needed; but two calls that may run at
+ *     the same time on the GPU (different streams, or different host threads) race on it: keep calls to this
+ *     entry point ordered on one stream, or serialise them yourself.
+ */
+#define PTQ_STATIC_SCRATCH_BYTES (6u << 20)
+int ptq_sensitivity_order_static(const float *W, int rows, int cols, int64_t ldw, const double *Hinv_diag,
+                                 const float *scale, const float *zero, int bits, int score_mode, double *S,
+                                 int32_t *perm, int32_t *status, void *stream);
 
 /*
  * Sec. 4.2 steps 3-5: permute W and Hinv by perm, then quantize one column at a time, all rows in parallel;

@@ -6,6 +6,8 @@
 #include "colloop.cuh"
 #include "gram.cuh"
 
+#include <mutex>
+
 using namespace ptq;
 
 namespace {
@@ -23,6 +25,31 @@ inline int grid_x_for(int n, int threads) {
 }
 
 size_t loss_partials_count(int rows, int cols) { return (size_t)cdiv(rows, 64) * cdiv(cols, 64); }
+
+// Built-in scratch of ptq_sensitivity_order_static: lives in every device that loads the library, until exit.
+constexpr size_t kStaticScratchDoubles = PTQ_STATIC_SCRATCH_BYTES / sizeof(double);
+static __device__ __align__(256) double g_static_score_scratch[kStaticScratchDoubles];
+
+// Device address of the array on the current device.  In host code the symbol's name is only a handle, so the
+// address is asked for once per device (with that device current) and remembered.
+int static_scratch_address(double** out) {
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static double* addr[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PTQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!addr[dev]) {
+        double* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_static_score_scratch) != cudaSuccess || !p) {
+            cudaGetLastError();
+            return PTQ_ERR_CUDA;
+        }
+        addr[dev] = p;
+    }
+    *out = addr[dev];
+    return PTQ_OK;
+}
 
 }  // namespace
 
@@ -78,6 +105,7 @@ const char* ptq_status_string(int code) {
         case PTQ_ERR_TIMEOUT: return "bounded device wait expired";
         case PTQ_ERR_CUDA: return "CUDA runtime error";
         case PTQ_ERR_UNSUPPORTED: return "unsupported configuration";
+        case PTQ_ERR_STATIC_SCRATCH: return "problem too large for the built-in scratch array";
         default: return "unknown status";
     }
 }
@@ -193,6 +221,31 @@ int ptq_sensitivity_order(const float* W, int rows, int cols, int64_t ldw, const
     Carver cv(ws);
     const int chunks = cdiv(rows, kScoreRowChunk);
     double* partial = cv.take<double>((size_t)chunks * cols);
+    if (score_mode != PTQ_SCORE_NONE) {
+        Launch l(K_SCORE_PARTIAL, stream);
+        score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
+                                                                              score_mode, partial);
+    }
+    { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status); }
+    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(S, cols, perm); }
+    return launch_status();
+}
+
+int ptq_sensitivity_order_static(const float* W, int rows, int cols, int64_t ldw, const double* Hinv_diag,
+                                 const float* scale, const float* zero, int bits, int score_mode, double* S,
+                                 int32_t* perm, int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!W || !S || !perm || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8) return PTQ_ERR_INVALID_ARG;
+    if (score_mode < PTQ_SCORE_QERR || score_mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
+    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_PRUNE) && !Hinv_diag) return PTQ_ERR_INVALID_ARG;
+    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_ERR) && (!scale || !zero)) return PTQ_ERR_INVALID_ARG;
+    const int chunks = cdiv(rows, kScoreRowChunk);
+    if ((size_t)chunks * (size_t)cols > kStaticScratchDoubles) return PTQ_ERR_STATIC_SCRATCH;
+    double* partial = nullptr;
+    const int st = static_scratch_address(&partial);
+    if (st) return st;
+    // Every partial[ch][j] that score_final_kernel reads is written first by score_partial_kernel, so nothing
+    // left in the array by an earlier call is ever used and nothing needs clearing.
     if (score_mode != PTQ_SCORE_NONE) {
         Launch l(K_SCORE_PARTIAL, stream);
         score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,

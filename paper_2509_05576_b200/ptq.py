@@ -16,12 +16,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libptq.so")
 
 OK, ERR_INVALID_ARG, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_NOT_SPD, ERR_NONFINITE, ERR_TIMEOUT, ERR_CUDA, ERR_UNSUPPORTED = range(9)
+ERR_STATIC_SCRATCH = 9
+STATIC_SCRATCH_BYTES = 6 << 20
 DAMP_REL_MEAN_DIAG, DAMP_ABS = 0, 1
 SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
 CALL_HESSIAN_ACCUMULATE, CALL_PREPARE_HINV, CALL_SENSITIVITY_ORDER, CALL_QUANTIZE_LAYER, CALL_HESSIAN_ACCUMULATE_F64 = range(5)
 
 EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
-           "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
+           "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_sensitivity_order_static", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
            "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
 
 
@@ -55,6 +57,7 @@ def lib():
         L.ptq_minmax_grid.argtypes = [vp, c_int, c_int, c_int64, c_int, vp, vp, vp, vp]
         L.ptq_sensitivity_order.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, c_size_t,
                                             vp, vp]
+        L.ptq_sensitivity_order_static.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, vp]
         L.ptq_quantize_layer.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, vp, c_int, vp, vp, vp, vp, vp,
                                          c_size_t, vp, vp]
         L.ptq_status_string.argtypes = [c_int]
@@ -191,6 +194,18 @@ def sensitivity_order(W, Hinv_diag, scale, zero, bits, score_mode, S, perm, ws, 
     _check(lib().ptq_sensitivity_order(_ptr(W), rows, cols, _rowmajor(W, "W"), _ptr(Hinv_diag), _ptr(scale),
                                        _ptr(zero), int(bits), int(score_mode), _ptr(S), _ptr(perm), _ptr(buf),
                                        buf.numel(), _ptr(status), _stream(stream)), "ptq_sensitivity_order")
+
+
+def sensitivity_order_static(W, Hinv_diag, scale, zero, bits, score_mode, S, perm, status, stream=None):
+    """``sensitivity_order`` without a workspace argument, for callers that may not allocate device memory: the
+    scratch is an array built into the library (``STATIC_SCRATCH_BYTES``).  Raises ``PtqError`` with
+    ``ERR_STATIC_SCRATCH`` when ceil(rows / 64) * cols * 8 bytes exceeds it.  Calls share that array, so keep them
+    ordered on one stream."""
+    _dev(W, torch.float32, "W")
+    rows, cols = W.shape
+    _check(lib().ptq_sensitivity_order_static(_ptr(W), rows, cols, _rowmajor(W, "W"), _ptr(Hinv_diag), _ptr(scale),
+                                              _ptr(zero), int(bits), int(score_mode), _ptr(S), _ptr(perm),
+                                              _ptr(status), _stream(stream)), "ptq_sensitivity_order_static")
 
 
 def quantize_layer(W, Hinv, perm, scale, zero, bits, codes, What, H_undamped, loss_out, ws, status, stream=None):
