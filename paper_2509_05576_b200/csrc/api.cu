@@ -126,6 +126,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
         case PTQ_CALL_PREPARE_HINV:
             add(c * c * sizeof(double));
             add(c * c * sizeof(double));
+            add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
             break;
         case PTQ_CALL_SENSITIVITY_ORDER:
             if (rows < 1) return 0;
@@ -140,6 +141,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(c * sizeof(int32_t));                       // flags
             add(c * sizeof(int32_t));                       // inverse permutation
             add(loss_partials_count(rows, cols) * sizeof(double));
+            add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
             break;
         default:
             return 0;
@@ -186,9 +188,10 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     Carver cv(ws);
     double* R = cv.take<double>((size_t)n * n);
     double* V = cv.take<double>((size_t)n * n);
+    unsigned* bar = cv.take<unsigned>(2);
     { Launch l(K_LAMBDA, stream); lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status); }
     { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out); }
-    int st = cholesky_upper(R, n, status, stream);
+    int st = cholesky_upper(R, n, bar, status, stream);
     if (st) return st;
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     st = trtri_upper(R, V, Hinv, n, stream);
@@ -280,6 +283,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     int32_t* flags = cv.take<int32_t>(n);
     int32_t* invperm = cv.take<int32_t>(n);
     double* partials = cv.take<double>(loss_partials_count(rows, cols));
+    unsigned* bar = cv.take<unsigned>(2);
 
     // flags and invperm are adjacent pieces of the workspace: clear both
     if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
@@ -288,7 +292,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     { Launch l(K_PERM_CHECK, stream); perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status); }
     { Launch l(K_GATHER_SYM, stream); gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U); }
     { Launch l(K_GATHER_W, stream); gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp); }
-    int st = cholesky_upper(U, n, status, stream);   // blocked Eq. 12
+    int st = cholesky_upper(U, n, bar, status, stream);   // blocked Eq. 12
     if (st) return st;
 
     const int row_ctas = cdiv(rows, kRowsPerCta);

@@ -5,6 +5,7 @@
 #pragma once
 #include "common.cuh"
 #include "dgemm.cuh"
+#include <utility>
 
 namespace ptq {
 
@@ -41,81 +42,256 @@ __global__ void damp_copy_kernel(const double* __restrict__ H, double* __restric
     }
 }
 
-// Upper Cholesky of the kb x kb diagonal block at (k0, k0), one CTA.  Row p of the factor is written to
-// global memory as soon as step p fixes it.  A non-positive or non-finite pivot is reported and replaced by 1.
-__global__ void __launch_bounds__(256) potrf_diag_kernel(double* __restrict__ A, int64_t ld, int k0, int kb,
-                                                          int32_t* status) {
-    __shared__ double S[kNB][kNB + 1];
-    const int tid = threadIdx.x;
-    for (int idx = tid; idx < kNB * kNB; idx += 256) {
-        const int r = idx >> 6, c = idx & 63;
-        double v = (r == c) ? 1.0 : 0.0;
-        if (r < kb && c < kb && c >= r) v = A[(int64_t)(k0 + r) * ld + k0 + c];
-        S[r][c] = v;
+// ------------------------------------------------------------------------------------------------------------
+// Blocked upper Cholesky A = U^T U as ONE persistent cooperative kernel (one CTA per SM, 256 threads).
+// For each 64-row block k:
+//   strip phase    every CTA that owns panel columns factorises the 64 x 64 diagonal block itself (all CTAs do the
+//                  same arithmetic on it, so no broadcast is needed) and applies the same row operations to its own
+//                  192 panel columns: one thread per column, the column's 64 entries in registers, row p of the
+//                  diagonal block broadcast through shared memory at step p.  That is the unblocked algorithm on a
+//                  64-row strip, and it replaces "factor the block, then solve the panel against it".
+//   trailing phase A[i][j] -= U[k][i]^T U[k][j] on the upper 64 x 64 tiles, float64 tensor-core MMA, operands
+//                  double-buffered through shared memory with cp.async.
+// The phases are separated by a grid-wide barrier whose wait is bounded: when it expires the CTA records
+// PTQ_ERR_TIMEOUT, raises the abort word and leaves; the other CTAs see the abort word and leave too.
+// A non-positive or non-finite pivot is reported (PTQ_ERR_NOT_SPD, pivot index) and replaced by 1.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kCholThreads = 256;
+constexpr int kCholPanelCols = kCholThreads - kNB;            // 192 panel columns per CTA in the strip phase
+constexpr int kCholLd = kNB + 4;                               // operand row stride (68 = 4 mod 16: conflict-free)
+constexpr size_t kCholSmemBytes = sizeof(double) * (2 * 2 * kNB * kCholLd + 2 * kNB) + 16;
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// bar[0]: arrival counter (monotonic, zero at launch), bar[1]: abort word.  Returns false when the CTA must leave.
+__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int* s_flag) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        atomicAdd(&bar[0], 1u);
+        const long long t0 = clock64();
+        int ok = 1;
+        unsigned it = 0;
+        while (ld_acquire_u32(&bar[0]) < target) {
+            if ((++it & 63u) == 0u) {
+                if (ld_acquire_u32(&bar[1]) != 0u) { ok = 0; break; }
+                if (clock64() - t0 > 4000000000LL) { atomicExch(&bar[1], 1u); ok = 0; break; }
+            }
+        }
+        __threadfence();
+        *s_flag = ok;
     }
     __syncthreads();
-    for (int p = 0; p < kNB; ++p) {
-        double d = S[p][p];
-        if (!(d > 0.0) || !isfinite(d)) {
-            if (tid == 0) report(status, PTQ_ERR_NOT_SPD, k0 + p);
-            d = 1.0;
+    return *s_flag != 0;
+}
+
+__device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gsrc, bool valid) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const int sz = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(sz) : "memory");
+}
+
+// Loads the 64 x 64 block A[r0 .. r0+63][c0 .. c0+63] into dst[64][kCholLd]; entries beyond n are zero.
+__device__ __forceinline__ void chol_load_block(double* dst, const double* __restrict__ A, int64_t ld, int n, int r0,
+                                                int c0, int vec16) {
+    if (vec16) {
+        for (int idx = threadIdx.x; idx < kNB * kNB / 2; idx += kCholThreads) {
+            const int r = idx >> 5, c = (idx & 31) * 2;
+            const bool ok = r0 + r < n && c0 + c < n;      // n is even on this path: a pair never straddles n
+            cp_async16_cg(dst + r * kCholLd + c, ok ? A + (int64_t)(r0 + r) * ld + c0 + c : A, ok);
         }
-        const double inv = 1.0 / d;
-        if (tid >= p && tid < kb && p < kb) A[(int64_t)(k0 + p) * ld + k0 + tid] = S[p][tid] / sqrt(d);
-        for (int idx = tid; idx < kNB * kNB; idx += 256) {
-            const int i = idx >> 6, j = idx & 63;
-            if (i > p && j >= i) S[i][j] -= S[p][i] * S[p][j] * inv;
+    } else {
+        for (int idx = threadIdx.x; idx < kNB * kNB; idx += kCholThreads) {
+            const int r = idx >> 6, c = idx & 63;
+            const bool ok = r0 + r < n && c0 + c < n;
+            cp_async8(dst + r * kCholLd + c, ok ? A + (int64_t)(r0 + r) * ld + c0 + c : A, ok);
         }
-        __syncthreads();
     }
 }
 
-// Row panel: U[k0:k0+kb, c] = U_kk^-T A[k0:k0+kb, c] for the columns c >= k0 + kb, one thread per column
-// (forward substitution against the transposed diagonal factor held in shared memory).
-__global__ void __launch_bounds__(128) panel_solve_kernel(double* __restrict__ A, int64_t ld, int k0, int kb, int n) {
-    __shared__ double Us[kNB][kNB];
-    for (int idx = threadIdx.x; idx < kNB * kNB; idx += 128) {
-        const int r = idx >> 6, c = idx & 63;
-        double v = (r == c) ? 1.0 : 0.0;
-        if (r < kb && c < kb && c >= r) v = A[(int64_t)(k0 + r) * ld + k0 + c];
-        Us[r][c] = v;
-    }
+// Step P of the strip factorisation: row P of the diagonal block is published, every thread scales its own entry
+// of that row and eliminates it from the rows below.
+template <int P>
+__device__ __forceinline__ void chol_strip_step(double (&col)[kNB], double* rowbuf, bool is_diag, int tid, int g,
+                                                int k0, int32_t* status) {
+    double* rb = rowbuf + (P & 1) * kNB;
+    if (is_diag) rb[tid] = col[P];
     __syncthreads();
-    const int col = k0 + kb + blockIdx.x * 128 + threadIdx.x;
-    if (col >= n) return;
-    double y[kNB];
-#pragma unroll
-    for (int r = 0; r < kNB; ++r) y[r] = (r < kb) ? A[(int64_t)(k0 + r) * ld + col] : 0.0;
-#pragma unroll
-    for (int r = 0; r < kNB; ++r) {
-        double s = y[r];
-#pragma unroll
-        for (int t = 0; t < r; ++t) s = fma(-Us[t][r], y[t], s);
-        y[r] = s / Us[r][r];
+    double d = rb[P];
+    if (!(d > 0.0) || !isfinite(d)) {
+        if (tid == 0 && g == 0) report(status, PTQ_ERR_NOT_SPD, k0 + P);
+        d = 1.0;
     }
+    const double inv = 1.0 / d;
+    const double t = col[P] * inv;
+    col[P] = col[P] * sqrt(inv);                                  // U[P][c]
 #pragma unroll
-    for (int r = 0; r < kNB; ++r)
-        if (r < kb) A[(int64_t)(k0 + r) * ld + col] = y[r];
+    for (int i = P + 1; i < kNB; ++i) col[i] = fma(-rb[i], t, col[i]);
+}
+template <int... Ps>
+__device__ __forceinline__ void chol_strip_steps(double (&col)[kNB], double* rowbuf, bool is_diag, int tid, int g,
+                                                 int k0, int32_t* status, std::integer_sequence<int, Ps...>) {
+    (chol_strip_step<Ps>(col, rowbuf, is_diag, tid, g, k0, status), ...);
 }
 
-// In-place blocked upper Cholesky of the n x n matrix A (only the upper triangle is read or written as a result).
-inline int cholesky_upper(double* A, int n, int32_t* status, cudaStream_t stream) {
-    for (int k0 = 0; k0 < n; k0 += kNB) {
-        const int kb = n - k0 < kNB ? n - k0 : kNB;
-        { Launch l(K_POTRF_DIAG, stream); potrf_diag_kernel<<<1, 256, 0, stream>>>(A, n, k0, kb, status); }
-        const int rest = n - k0 - kb;
-        if (rest <= 0) break;
-        { Launch l(K_PANEL_SOLVE, stream); panel_solve_kernel<<<cdiv(rest, 128), 128, 0, stream>>>(A, n, k0, kb, n); }
-        GemmParams g = gemm_defaults();     // A22 -= U12^T U12 on the upper tiles
-        g.A = A + (int64_t)k0 * n + k0 + kb; g.lda = n; g.a_trans = 1;
-        g.B = g.A; g.ldb = n; g.b_trans = 0;
-        g.C = A + (int64_t)(k0 + kb) * n + k0 + kb; g.ldc = n;
-        g.M = rest; g.N = rest; g.K = kb;
-        g.alpha = -1.0; g.beta = 1.0; g.upper_only = 1;
-        int st = launch_dgemm(K_DGEMM_CHOL, g, 1, stream);
-        if (st) return st;
+__global__ void __launch_bounds__(kCholThreads, 1)
+chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned* bar, int32_t* status) {
+    extern __shared__ __align__(16) unsigned char chol_smem_raw[];
+    double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
+    double* rowbuf = opnd + 2 * 2 * kNB * kCholLd;                          // [2][64]
+    int* s_flag = reinterpret_cast<int*>(rowbuf + 2 * kNB);
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int G = gridDim.x;
+    const int nb = (n + kNB - 1) / kNB;
+    unsigned epoch = 0;
+
+    for (int k = 0; k < nb; ++k) {
+        const int k0 = k * kNB;
+        // ------------------------------------------------------------------ strip phase
+        const int panel_cols = n - k0 - kNB;                                // columns to the right of the block
+        const int groups = panel_cols > 0 ? (panel_cols + kCholPanelCols - 1) / kCholPanelCols : 0;
+        const int reps = groups > 0 ? groups : 1;                            // last block: diagonal only
+        for (int g = blockIdx.x; g < reps; g += G) {
+            // column owned by this thread: tid < 64 -> diagonal block column tid, else a panel column
+            const bool is_diag = tid < kNB;
+            const int gc = is_diag ? k0 + tid : k0 + kNB + g * kCholPanelCols + (tid - kNB);
+            const bool live = gc < n && (is_diag || groups > 0);
+            double col[kNB];
+#pragma unroll
+            for (int p = 0; p < kNB; ++p) {
+                double v = (is_diag && p == tid) ? 1.0 : 0.0;                // identity padding below n
+                if (live && k0 + p < n && (!is_diag || p <= tid)) v = __ldcg(A + (int64_t)(k0 + p) * ld + gc);
+                col[p] = v;
+            }
+            chol_strip_steps(col, rowbuf, is_diag, tid, g, k0, status, std::make_integer_sequence<int, kNB>());
+            if (live) {
+                if (is_diag) {
+                    if (g == 0) {
+#pragma unroll
+                        for (int p = 0; p < kNB; ++p)
+                            if (p <= tid && k0 + p < n) __stcg(A + (int64_t)(k0 + p) * ld + gc, col[p]);
+                    }
+                } else {
+#pragma unroll
+                    for (int p = 0; p < kNB; ++p)
+                        if (k0 + p < n) __stcg(A + (int64_t)(k0 + p) * ld + gc, col[p]);
+                }
+            }
+            __syncthreads();     // rowbuf is reused by the next repetition
+        }
+        if (k == nb - 1) break;
+        ++epoch;
+        if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
+
+        // ------------------------------------------------------------------ trailing phase
+        const int m = nb - 1 - k;
+        const int T = m * (m + 1) / 2;
+        auto tile_ij = [&](int t, int& bi, int& bj) {
+            int i = k + 1, rem = t;
+            while (rem >= nb - i) { rem -= nb - i; ++i; }
+            bi = i; bj = i + rem;
+        };
+        int stage = 0;
+        if ((int)blockIdx.x < T) {
+            int bi, bj;
+            tile_ij(blockIdx.x, bi, bj);
+            chol_load_block(opnd, A, ld, n, k0, bi * kNB, vec16);
+            chol_load_block(opnd + kNB * kCholLd, A, ld, n, k0, bj * kNB, vec16);
+        }
+        cp_async_commit();
+        for (int t = blockIdx.x; t < T; t += G) {
+            int bi, bj;
+            tile_ij(t, bi, bj);
+            if (t + G < T) {
+                int ni, nj;
+                tile_ij(t + G, ni, nj);
+                double* nxt = opnd + (stage ^ 1) * 2 * kNB * kCholLd;
+                chol_load_block(nxt, A, ld, n, k0, ni * kNB, vec16);
+                chol_load_block(nxt + kNB * kCholLd, A, ld, n, k0, nj * kNB, vec16);
+            }
+            cp_async_commit();
+            cp_async_wait<1>();
+            __syncthreads();
+            const double* as = opnd + stage * 2 * kNB * kCholLd;            // as[kk][m] = U[k0 + kk][i0 + m]
+            const double* bs = as + kNB * kCholLd;                           // bs[kk][n] = U[k0 + kk][j0 + n]
+            const int wm0 = (warp >> 2) * 32, wn0 = (warp & 3) * 16;
+            const int lq = lane >> 2, lr = lane & 3;
+            double acc[4][2][2];
+#pragma unroll
+            for (int a = 0; a < 4; ++a)
+#pragma unroll
+                for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
+#pragma unroll 4
+            for (int kk = 0; kk < kNB; kk += 4) {
+                double af[4], bf[2];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) af[a] = as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
+#pragma unroll
+                for (int b = 0; b < 2; ++b) bf[b] = bs[(kk + lr) * kCholLd + wn0 + b * 8 + lq];
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int b = 0; b < 2; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+            }
+            const int i0 = bi * kNB, j0 = bj * kNB;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+                const int r = wm0 + a * 8 + lq;
+#pragma unroll
+                for (int b = 0; b < 2; ++b)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int c = wn0 + b * 8 + 2 * lr + e;
+                        if (i0 + r < n && j0 + c < n && (bi != bj || c >= r)) {
+                            double* dst = A + (int64_t)(i0 + r) * ld + j0 + c;
+                            __stcg(dst, __ldcg(dst) - acc[a][b][e]);
+                        }
+                    }
+            }
+            __syncthreads();     // all warps are done with this stage before it is refilled
+            stage ^= 1;
+        }
+        cp_async_wait<0>();
+        ++epoch;
+        if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
     }
-    return launch_status();
+    cp_async_wait<0>();
+    if (tid == 0 && ld_acquire_u32(&bar[1]) != 0u) report(status, PTQ_ERR_TIMEOUT, blockIdx.x, 1);
+}
+
+// In-place blocked upper Cholesky of the n x n matrix A (row stride n).  Only the upper triangle is read or
+// written.  `bar` is 2 x uint32 of device scratch.
+inline int cholesky_upper(double* A, int n, unsigned* bar, int32_t* status, cudaStream_t stream) {
+    static int grid = 0;
+    if (grid == 0) {
+        if (cudaFuncSetAttribute(chol_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)kCholSmemBytes) != cudaSuccess)
+            return PTQ_ERR_CUDA;
+        int dev = 0, sms = 0, per_sm = 0, coop = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+        if (!coop) return PTQ_ERR_UNSUPPORTED;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chol_coop_kernel, kCholThreads, kCholSmemBytes) !=
+                cudaSuccess || per_sm < 1)
+            return PTQ_ERR_CUDA;
+        grid = sms;          // one CTA per SM: the cooperative launch guarantees that all of them are resident
+    }
+    if (cudaMemsetAsync(bar, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
+    int64_t ld = n;
+    int vec16 = ((n & 1) == 0 && aligned16(A)) ? 1 : 0;
+    void* args[] = {&A, &n, &ld, &vec16, &bar, &status};
+    Launch l(K_CHOL_COOP, stream);
+    if (cudaLaunchCooperativeKernel((const void*)chol_coop_kernel, dim3(grid), dim3(kCholThreads), args,
+                                    kCholSmemBytes, stream) != cudaSuccess) {
+        cudaGetLastError();
+        return PTQ_ERR_CUDA;
+    }
+    return PTQ_OK;
 }
 
 // V[b, b] = inverse of the upper-triangular diagonal block R[b, b]; one CTA per 64-block, one thread per column.

@@ -1,7 +1,8 @@
-// Float64 GEMM tile kernel used by every float64 stage: the Cholesky trailing updates, the triangular
-// inverse, Hinv = V V^T, the deferred Eq.-11 update of W, the float64 cross-check Gram and the loss
-// 1/2 tr(dW H dW^T).  One kernel, parameterised by operand layout and by the triangular structure it
-// may exploit.  All sums run over k in ascending order inside a tile, so results are deterministic.
+// Float64 GEMM tile kernel used by every float64 stage: the triangular inverse, Hinv = V V^T, the float64
+// cross-check Gram and the loss 1/2 tr(dW H dW^T).  One kernel, parameterised by operand layout and by the
+// triangular structure it may exploit.  The products run on the float64 tensor-core instruction
+// (mma.sync m8n8k4), operands are staged through shared memory by a 3-stage cp.async pipeline.
+// All sums run over k in ascending order, so results are deterministic.
 #pragma once
 #include "common.cuh"
 
@@ -30,22 +31,40 @@ struct GemmParams {
 };
 
 constexpr int kGemmBK = 16;
+constexpr int kGemmStages = 3;
 constexpr int kGemmThreads = 256;
+constexpr int kGemmLdk = kGemmBK + 4;   // row stride of a k-contiguous operand tile (20 = 4 mod 16: conflict-free)
 
 template <int BT>
-constexpr size_t gemm_smem_bytes() { return size_t(2) * 2 * kGemmBK * (BT + 2) * sizeof(double); }
+constexpr int gemm_tile_doubles() { return BT * kGemmLdk; }   // >= 16 * (BT + 4), the m-contiguous layout
+template <int BT>
+constexpr size_t gemm_smem_bytes() { return size_t(kGemmStages) * 2 * gemm_tile_doubles<BT>() * sizeof(double); }
 
-// BT x BT output tile, 256 threads, each thread owns (BT/16) x (BT/16) outputs as 2-wide groups spaced 32 apart.
+__device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc, bool valid) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const int sz = valid ? 8 : 0;    // src-size 0: the 8 bytes are filled with zeros
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(d), "l"(gsrc), "r"(sz) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__device__ __forceinline__ void dmma_884(double& c0, double& c1, double a, double b) {
+    asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
+                 : "+d"(c0), "+d"(c1)
+                 : "d"(a), "d"(b));
+}
+
+// BT x BT output tile, 256 threads = 8 warps as 2 x 4; each warp owns (BT/2) x (BT/4) outputs as 8 x 8 fragments.
 template <int BT>
 __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
     constexpr int BK = kGemmBK;
-    constexpr int LD = BT + 2;
-    constexpr int T = BT / 16;        // outputs per thread per dimension
-    constexpr int G = T / 2;          // 2-wide groups per dimension
-    constexpr int EPT = BT * BK / kGemmThreads;  // elements each thread stages per operand tile
+    constexpr int LDM = BT + 4;            // row stride of an m-contiguous operand tile
+    constexpr int TILE = BT * kGemmLdk;
+    constexpr int WTM = BT / 2, WTN = BT / 4;
+    constexpr int FM = WTM / 8, FN = WTN / 8;
+    constexpr int EPT = BT * BK / kGemmThreads;
     extern __shared__ __align__(16) double smem[];
-    double* As = smem;                    // [2][BK][LD]
-    double* Bs = smem + 2 * BK * LD;      // [2][BK][LD]
 
     const int z = blockIdx.z;
     int N = p.N, K = p.K;
@@ -70,101 +89,89 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
     kbeg = (kbeg / BK) * BK;
     if (p.kend_mode == 1 && j0 + BT < kend) kend = j0 + BT;
 
-    const int tid = threadIdx.x;
-    const int tx = tid & 15, ty = tid >> 4;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int wm0 = (warp >> 2) * WTM, wn0 = (warp & 3) * WTN;
+    const int lq = lane >> 2, lr = lane & 3;
+    const int a_trans = p.a_trans, b_trans = p.b_trans;
 
-    double acc[T][T];
+    double acc[FM][FN][2];
 #pragma unroll
-    for (int a = 0; a < T; ++a)
+    for (int a = 0; a < FM; ++a)
 #pragma unroll
-        for (int b = 0; b < T; ++b) acc[a][b] = 0.0;
+        for (int b = 0; b < FN; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
 
-    double ra[EPT], rb[EPT];
-
-    auto load_tiles = [&](int k0) {
+    auto load_stage = [&](int stage, int k0) {
+        double* as = smem + (size_t)stage * 2 * TILE;
+        double* bs = as + TILE;
 #pragma unroll
         for (int r = 0; r < EPT; ++r) {
-            int i, k;
-            if (p.a_trans == 0) { k = tid & 15; i = (tid >> 4) + 16 * r; }
-            else { i = tid % BT; k = tid / BT + (kGemmThreads / BT) * r; }
-            const int gi = i0 + i, gk = k0 + k;
-            double v = 0.0;
-            if (gi < M && gk < kend)
-                v = p.a_trans == 0 ? A[(int64_t)gi * p.lda + gk] : A[(int64_t)gk * p.lda + gi];
-            ra[r] = v;
+            const int idx = tid + r * kGemmThreads;
+            int m, k, off;
+            if (a_trans == 0) { k = idx & 15; m = idx >> 4; off = m * kGemmLdk + k; }
+            else { m = idx % BT; k = idx / BT; off = k * LDM + m; }
+            const int gi = i0 + m, gk = k0 + k;
+            const bool ok = gi < M && gk < kend;
+            const double* src = ok ? (a_trans == 0 ? A + (int64_t)gi * p.lda + gk : A + (int64_t)gk * p.lda + gi) : A;
+            cp_async8(as + off, src, ok);
         }
 #pragma unroll
         for (int r = 0; r < EPT; ++r) {
-            int j, k;
-            if (p.b_trans == 1) { k = tid & 15; j = (tid >> 4) + 16 * r; }
-            else { j = tid % BT; k = tid / BT + (kGemmThreads / BT) * r; }
-            const int gj = j0 + j, gk = k0 + k;
-            double v = 0.0;
-            if (gj < N && gk < kend)
-                v = p.b_trans == 1 ? B[(int64_t)gj * p.ldb + gk] : B[(int64_t)gk * p.ldb + gj];
-            rb[r] = v;
-        }
-    };
-    auto store_tiles = [&](int buf) {
-        double* as = As + buf * BK * LD;
-        double* bs = Bs + buf * BK * LD;
-#pragma unroll
-        for (int r = 0; r < EPT; ++r) {
-            int i, k;
-            if (p.a_trans == 0) { k = tid & 15; i = (tid >> 4) + 16 * r; }
-            else { i = tid % BT; k = tid / BT + (kGemmThreads / BT) * r; }
-            as[k * LD + i] = ra[r];
-        }
-#pragma unroll
-        for (int r = 0; r < EPT; ++r) {
-            int j, k;
-            if (p.b_trans == 1) { k = tid & 15; j = (tid >> 4) + 16 * r; }
-            else { j = tid % BT; k = tid / BT + (kGemmThreads / BT) * r; }
-            bs[k * LD + j] = rb[r];
+            const int idx = tid + r * kGemmThreads;
+            int n, k, off;
+            if (b_trans == 1) { k = idx & 15; n = idx >> 4; off = n * kGemmLdk + k; }
+            else { n = idx % BT; k = idx / BT; off = k * LDM + n; }
+            const int gj = j0 + n, gk = k0 + k;
+            const bool ok = gj < N && gk < kend;
+            const double* src = ok ? (b_trans == 1 ? B + (int64_t)gj * p.ldb + gk : B + (int64_t)gk * p.ldb + gj) : B;
+            cp_async8(bs + off, src, ok);
         }
     };
 
-    if (kbeg < kend) {
-        load_tiles(kbeg);
-        store_tiles(0);
+    const int nkt = kbeg < kend ? (kend - kbeg + BK - 1) / BK : 0;
+    // element (m, k) of the A tile and (k, n) of the B tile, in doubles
+    const int a_sm = a_trans == 0 ? kGemmLdk : 1, a_sk = a_trans == 0 ? 1 : LDM;
+    const int b_sn = b_trans == 1 ? kGemmLdk : 1, b_sk = b_trans == 1 ? 1 : LDM;
+    const int a_lane = (wm0 + lq) * a_sm + lr * a_sk;
+    const int b_lane = (wn0 + lq) * b_sn + lr * b_sk;
+
+    for (int s = 0; s < kGemmStages - 1; ++s) {
+        if (s < nkt) load_stage(s, kbeg + s * BK);
+        cp_async_commit();
+    }
+    for (int kt = 0; kt < nkt; ++kt) {
+        cp_async_wait<kGemmStages - 2>();
         __syncthreads();
-        int buf = 0;
-        for (int k0 = kbeg; k0 < kend; k0 += BK) {
-            const bool more = k0 + BK < kend;
-            if (more) load_tiles(k0 + BK);
-            const double* as = As + buf * BK * LD;
-            const double* bs = Bs + buf * BK * LD;
+        if (kt + kGemmStages - 1 < nkt) load_stage((kt + kGemmStages - 1) % kGemmStages, kbeg + (kt + kGemmStages - 1) * BK);
+        cp_async_commit();
+        const double* as = smem + (size_t)(kt % kGemmStages) * 2 * TILE;
+        const double* bs = as + TILE;
 #pragma unroll
-            for (int k = 0; k < BK; ++k) {
-                double av[T], bv[T];
+        for (int kk = 0; kk < BK; kk += 4) {
+            double af[FM], bf[FN];
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const double2 a2 = *reinterpret_cast<const double2*>(as + k * LD + g * 32 + ty * 2);
-                    const double2 b2 = *reinterpret_cast<const double2*>(bs + k * LD + g * 32 + tx * 2);
-                    av[2 * g] = a2.x; av[2 * g + 1] = a2.y;
-                    bv[2 * g] = b2.x; bv[2 * g + 1] = b2.y;
-                }
+            for (int a = 0; a < FM; ++a) af[a] = as[a_lane + a * 8 * a_sm + kk * a_sk];
 #pragma unroll
-                for (int a = 0; a < T; ++a)
+            for (int b = 0; b < FN; ++b) bf[b] = bs[b_lane + b * 8 * b_sn + kk * b_sk];
 #pragma unroll
-                    for (int b = 0; b < T; ++b) acc[a][b] = fma(av[a], bv[b], acc[a][b]);
-            }
-            if (more) store_tiles(buf ^ 1);
-            __syncthreads();
-            buf ^= 1;
+            for (int a = 0; a < FM; ++a)
+#pragma unroll
+                for (int b = 0; b < FN; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
         }
     }
+    cp_async_wait<0>();
 
     if (p.partials) {
         double s = 0.0;
 #pragma unroll
-        for (int a = 0; a < T; ++a) {
-            const int gi = i0 + (a >> 1) * 32 + ty * 2 + (a & 1);
+        for (int a = 0; a < FM; ++a) {
+            const int gi = i0 + wm0 + a * 8 + lq;
 #pragma unroll
-            for (int b = 0; b < T; ++b) {
-                const int gj = j0 + (b >> 1) * 32 + tx * 2 + (b & 1);
-                if (gi < M && gj < N) s = fma(acc[a][b], p.D[(int64_t)gi * p.ldd + gj], s);
-            }
+            for (int b = 0; b < FN; ++b)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int gj = j0 + wn0 + b * 8 + 2 * lr + e;
+                    if (gi < M && gj < N) s = fma(acc[a][b][e], p.D[(int64_t)gi * p.ldd + gj], s);
+                }
         }
         __syncthreads();
         double* red = smem;
@@ -181,18 +188,20 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
 
     const bool do_mirror = p.mirror && (i0 != j0);
 #pragma unroll
-    for (int a = 0; a < T; ++a) {
-        const int gi = i0 + (a >> 1) * 32 + ty * 2 + (a & 1);
+    for (int a = 0; a < FM; ++a) {
+        const int gi = i0 + wm0 + a * 8 + lq;
         if (gi >= M) continue;
 #pragma unroll
-        for (int b = 0; b < T; ++b) {
-            const int gj = j0 + (b >> 1) * 32 + tx * 2 + (b & 1);
-            if (gj >= N) continue;
-            double v = p.alpha * acc[a][b];
-            if (p.beta != 0.0) v = fma(p.beta, C[(int64_t)gi * p.ldc + gj], v);
-            C[(int64_t)gi * p.ldc + gj] = v;
-            if (do_mirror) C[(int64_t)gj * p.ldc + gi] = v;
-        }
+        for (int b = 0; b < FN; ++b)
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int gj = j0 + wn0 + b * 8 + 2 * lr + e;
+                if (gj >= N) continue;
+                double v = p.alpha * acc[a][b][e];
+                if (p.beta != 0.0) v = fma(p.beta, C[(int64_t)gi * p.ldc + gj], v);
+                C[(int64_t)gi * p.ldc + gj] = v;
+                if (do_mirror) C[(int64_t)gj * p.ldc + gi] = v;
+            }
     }
 }
 
