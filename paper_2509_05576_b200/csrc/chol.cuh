@@ -45,11 +45,10 @@ __global__ void damp_copy_kernel(const double* __restrict__ H, double* __restric
 // ------------------------------------------------------------------------------------------------------------
 // Blocked upper Cholesky A = U^T U as ONE persistent cooperative kernel (one CTA per SM, 256 threads).
 // For each 64-row block k:
-//   strip phase    every CTA that owns panel columns factorises the 64 x 64 diagonal block itself (all CTAs do the
-//                  same arithmetic on it, so no broadcast is needed) and applies the same row operations to its own
-//                  192 panel columns: one thread per column, the column's 64 entries in registers, row p of the
-//                  diagonal block broadcast through shared memory at step p.  That is the unblocked algorithm on a
-//                  64-row strip, and it replaces "factor the block, then solve the panel against it".
+//   strip phase    every CTA that owns a 64-column panel chunk factorises the 64 x 64 diagonal block itself (all
+//                  CTAs do the same arithmetic on it, so no broadcast is needed) and applies the same row
+//                  operations to its chunk: the unblocked algorithm on a 64 x 128 strip, eight pivots at a time
+//                  (see chol_strip).  That replaces "factor the block, then solve the panel against it".
 //   trailing phase A[i][j] -= U[k][i]^T U[k][j] on the upper 64 x 64 tiles, float64 tensor-core MMA, operands
 //                  double-buffered through shared memory with cp.async.
 // The phases are separated by a grid-wide barrier whose wait is bounded: when it expires the CTA records
@@ -57,9 +56,8 @@ __global__ void damp_copy_kernel(const double* __restrict__ H, double* __restric
 // A non-positive or non-finite pivot is reported (PTQ_ERR_NOT_SPD, pivot index) and replaced by 1.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kCholThreads = 256;
-constexpr int kCholPanelCols = kCholThreads - kNB;            // 192 panel columns per CTA in the strip phase
 constexpr int kCholLd = kNB + 4;                               // operand row stride (68 = 4 mod 16: conflict-free)
-constexpr size_t kCholSmemBytes = sizeof(double) * (2 * 2 * kNB * kCholLd + 2 * kNB) + 16;
+constexpr size_t kCholSmemBytes = sizeof(double) * (2 * 2 * kNB * kCholLd) + 16;
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     unsigned v;
@@ -95,56 +93,230 @@ __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gsrc, 
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(sz) : "memory");
 }
 
-// Loads the 64 x 64 block A[r0 .. r0+63][c0 .. c0+63] into dst[64][kCholLd]; entries beyond n are zero.
+// Loads the 64 x ncols block A[r0 .. r0+63][c0 .. c0+ncols-1] into dst[64][kCholLd]; entries beyond n are zero.
 __device__ __forceinline__ void chol_load_block(double* dst, const double* __restrict__ A, int64_t ld, int n, int r0,
-                                                int c0, int vec16) {
+                                                int c0, int ncols, int vec16) {
     if (vec16) {
         for (int idx = threadIdx.x; idx < kNB * kNB / 2; idx += kCholThreads) {
             const int r = idx >> 5, c = (idx & 31) * 2;
+            if (c >= ncols) continue;
             const bool ok = r0 + r < n && c0 + c < n;      // n is even on this path: a pair never straddles n
             cp_async16_cg(dst + r * kCholLd + c, ok ? A + (int64_t)(r0 + r) * ld + c0 + c : A, ok);
         }
     } else {
         for (int idx = threadIdx.x; idx < kNB * kNB; idx += kCholThreads) {
             const int r = idx >> 6, c = idx & 63;
+            if (c >= ncols) continue;
             const bool ok = r0 + r < n && c0 + c < n;
             cp_async8(dst + r * kCholLd + c, ok ? A + (int64_t)(r0 + r) * ld + c0 + c : A, ok);
         }
     }
 }
 
-// Step P of the strip factorisation: row P of the diagonal block is published, every thread scales its own entry
-// of that row and eliminates it from the rows below.
-template <int P>
-__device__ __forceinline__ void chol_strip_step(double (&col)[kNB], double* rowbuf, bool is_diag, int tid, int g,
-                                                int k0, int32_t* status) {
-    double* rb = rowbuf + (P & 1) * kNB;
-    if (is_diag) rb[tid] = col[P];
-    __syncthreads();
-    double d = rb[P];
-    if (!(d > 0.0) || !isfinite(d)) {
-        if (tid == 0 && g == 0) report(status, PTQ_ERR_NOT_SPD, k0 + P);
-        d = 1.0;
-    }
-    const double inv = 1.0 / d;
-    const double t = col[P] * inv;
-    col[P] = col[P] * sqrt(inv);                                  // U[P][c]
+// ------------------------------------------------------------------------------------------------------------
+// Strip factorisation: the 64 x 128 strip [diagonal block | 64 panel columns] is held in registers as 8 x 8
+// MMA accumulator fragments (warp w owns strip columns 16 w .. 16 w + 15, all 64 rows).  Pivots are taken eight
+// at a time.  For pivot block b:
+//   1. every warp publishes its piece of rows 8 b .. 8 b + 7 (the row panel R) to shared memory;
+//   2. every warp factorises the 8 x 8 diagonal mini-block M = U_M^T U_M redundantly, one column per lane with
+//      warp shuffles, and carries the identity along to obtain W = U_M^-T;
+//   3. the new rows U[8 b .. 8 b + 7][:] = W R come from two MMAs per fragment;
+//   4. they are published and subtracted from the rows below, A[i][c] -= U[p][i] U[p][c], again by MMA.
+// Two block-wide barriers per eight pivots; the only serial chain is the eight reciprocal square roots of step 2.
+// ------------------------------------------------------------------------------------------------------------
+constexpr int kStripLd = 132;                                            // row stride of the 8-row panels
+constexpr int kStripSmemDoubles = 2 * 8 * kStripLd + (kCholThreads / 32) * 64;
+static_assert(kStripSmemDoubles <= 2 * 2 * kNB * kCholLd, "the strip panels alias the trailing-phase operand buffers");
+
+__device__ __forceinline__ double shfl_f64(double x, int src) { return __shfl_sync(0xffffffffu, x, src); }
+
+template <int B>
+__device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
+                                                 int warp, int lane, int k0, bool reporter, int32_t* status) {
+    const int lq = lane >> 2, lr = lane & 3;
+    const int c0 = 16 * warp;
+    // 1. publish the row panel
 #pragma unroll
-    for (int i = P + 1; i < kNB; ++i) col[i] = fma(-rb[i], t, col[i]);
+    for (int cb = 0; cb < 2; ++cb)
+        *reinterpret_cast<double2*>(Rbuf + lq * kStripLd + c0 + 8 * cb + 2 * lr) =
+            make_double2(acc[B][cb][0], acc[B][cb][1]);
+    __syncthreads();
+    // 2. mini-block factorisation: lanes 0..7 own the columns of M, lanes 8..15 the columns of the identity
+    const int jj = lane & 15;
+    double v[8];
+#pragma unroll
+    for (int p = 0; p < 8; ++p)
+        v[p] = jj < 8 ? Rbuf[p * kStripLd + 8 * B + jj] : (p == jj - 8 ? 1.0 : 0.0);
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        const double x = v[p];
+        double d = shfl_f64(x, p);
+        if (!(d > 0.0) || !isfinite(d)) {
+            if (reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + p);
+            d = 1.0;
+        }
+        const double rs = rsqrt(d);
+        const double t = x * (rs * rs);
+        v[p] = x * rs;
+#pragma unroll
+        for (int i = p + 1; i < 8; ++i) v[i] = fma(-shfl_f64(x, i), t, v[i]);
+    }
+    double* wb = Wbuf + warp * 64;
+    if (lane >= 8 && lane < 16) {
+#pragma unroll
+        for (int p = 0; p < 8; ++p) wb[p * 8 + (lane - 8)] = v[p];      // W[p][j] = (U_M^-T)[p][j]
+    }
+    __syncwarp();
+    // 3. new rows = W R
+    const double a0 = wb[lq * 8 + lr], a1 = wb[lq * 8 + 4 + lr];
+#pragma unroll
+    for (int cb = 0; cb < 2; ++cb) {
+        const double b0 = Rbuf[lr * kStripLd + c0 + 8 * cb + lq];
+        const double b1 = Rbuf[(4 + lr) * kStripLd + c0 + 8 * cb + lq];
+        double r0 = 0.0, r1 = 0.0;
+        dmma_884(r0, r1, a0, b0);
+        dmma_884(r0, r1, a1, b1);
+        acc[B][cb][0] = r0;
+        acc[B][cb][1] = r1;
+        *reinterpret_cast<double2*>(Ubuf + lq * kStripLd + c0 + 8 * cb + 2 * lr) = make_double2(r0, r1);
+    }
+    __syncthreads();
+    // 4. rows below: acc[r] -= U[:, 8 r .. 8 r + 7]^T U[:, own columns]
+    if constexpr (B < 7) {
+        double bf[2][2];
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+            bf[cb][0] = Ubuf[lr * kStripLd + c0 + 8 * cb + lq];
+            bf[cb][1] = Ubuf[(4 + lr) * kStripLd + c0 + 8 * cb + lq];
+        }
+#pragma unroll
+        for (int r = B + 1; r < 8; ++r) {
+            const double n0 = -Ubuf[lr * kStripLd + 8 * r + lq];
+            const double n1 = -Ubuf[(4 + lr) * kStripLd + 8 * r + lq];
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                dmma_884(acc[r][cb][0], acc[r][cb][1], n0, bf[cb][0]);
+                dmma_884(acc[r][cb][0], acc[r][cb][1], n1, bf[cb][1]);
+            }
+        }
+    }
 }
-template <int... Ps>
-__device__ __forceinline__ void chol_strip_steps(double (&col)[kNB], double* rowbuf, bool is_diag, int tid, int g,
-                                                 int k0, int32_t* status, std::integer_sequence<int, Ps...>) {
-    (chol_strip_step<Ps>(col, rowbuf, is_diag, tid, g, k0, status), ...);
+template <int... Bs>
+__device__ __forceinline__ void chol_strip_blocks(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
+                                                  int warp, int lane, int k0, bool reporter, int32_t* status,
+                                                  std::integer_sequence<int, Bs...>) {
+    (chol_strip_block<Bs>(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, reporter, status), ...);
+}
+
+// Factorises the diagonal block at k0 and, when chunk >= 0, the 64 panel columns starting at
+// k0 + 64 + 64 * chunk with it.  The diagonal factor is written only when write_diag is set.
+__device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, int n, int k0, int chunk,
+                                           bool write_diag, double* smem, int vec16, int32_t* status) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lq = lane >> 2, lr = lane & 3;
+    double* Rbuf = smem;
+    double* Ubuf = smem + 8 * kStripLd;
+    double* Wbuf = smem + 2 * 8 * kStripLd;
+    const bool is_diag = warp < 4;
+    const int gc0 = is_diag ? k0 + 16 * warp : k0 + kNB + chunk * kNB + 16 * (warp - 4);   // first global column
+    const int sc0 = 16 * warp;                                                               // first strip column
+    double acc[8][2][2];
+#pragma unroll
+    for (int rb = 0; rb < 8; ++rb)
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+            const int row = 8 * rb + lq, grow = k0 + row;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int sc = sc0 + 8 * cb + 2 * lr + e, gc = gc0 + 8 * cb + 2 * lr + e;
+                double val = 0.0;
+                if (is_diag) {
+                    if (sc >= row) {
+                        if (grow < n && gc < n) val = __ldcg(A + (int64_t)grow * ld + gc);
+                        else if (sc == row) val = 1.0;                   // identity padding below n
+                    }
+                } else if (chunk >= 0 && grow < n && gc < n) {
+                    val = __ldcg(A + (int64_t)grow * ld + gc);
+                }
+                acc[rb][cb][e] = val;
+            }
+        }
+    chol_strip_blocks(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, write_diag && threadIdx.x == 0, status,
+                      std::make_integer_sequence<int, 8>());
+    if (is_diag ? write_diag : chunk >= 0) {
+#pragma unroll
+        for (int rb = 0; rb < 8; ++rb)
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const int row = 8 * rb + lq, grow = k0 + row;
+                const int sc = sc0 + 8 * cb + 2 * lr, gc = gc0 + 8 * cb + 2 * lr;
+                if (grow >= n || gc >= n) continue;
+                double* dst = A + (int64_t)grow * ld + gc;
+                const bool keep0 = !is_diag || sc >= row, keep1 = !is_diag || sc + 1 >= row;
+                if (vec16 && keep0) {
+                    __stcg(reinterpret_cast<double2*>(dst), make_double2(acc[rb][cb][0], acc[rb][cb][1]));
+                } else {
+                    if (keep0) __stcg(dst, acc[rb][cb][0]);
+                    if (keep1 && gc + 1 < n) __stcg(dst + 1, acc[rb][cb][1]);
+                }
+            }
+    }
+}
+
+// One H x 64 piece of a trailing tile: rows [h0, h0 + H) of tile (bi, bj), operands in shared memory.
+template <int H>
+__device__ __forceinline__ void chol_trailing_piece(double* __restrict__ A, int64_t ld, int n, const double* as,
+                                                    const double* bs, int bi, int bj, int h0, int vec16) {
+    constexpr int FM = H / 16;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int wm0 = (warp >> 2) * (H / 2), wn0 = (warp & 3) * 16;
+    const int lq = lane >> 2, lr = lane & 3;
+    double acc[FM][2][2];
+#pragma unroll
+    for (int a = 0; a < FM; ++a)
+#pragma unroll
+        for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
+#pragma unroll 4
+    for (int kk = 0; kk < kNB; kk += 4) {
+        double af[FM], bf[2];
+#pragma unroll
+        for (int a = 0; a < FM; ++a) af[a] = as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
+#pragma unroll
+        for (int b = 0; b < 2; ++b) bf[b] = bs[(kk + lr) * kCholLd + wn0 + b * 8 + lq];
+#pragma unroll
+        for (int a = 0; a < FM; ++a)
+#pragma unroll
+            for (int b = 0; b < 2; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+    }
+    const int i0 = bi * kNB + h0, j0 = bj * kNB;
+#pragma unroll
+    for (int a = 0; a < FM; ++a) {
+        const int r = wm0 + a * 8 + lq;
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+            const int c = wn0 + b * 8 + 2 * lr;
+            if (i0 + r >= n || j0 + c >= n) continue;
+            double* dst = A + (int64_t)(i0 + r) * ld + j0 + c;
+            const bool keep0 = bi != bj || c >= h0 + r, keep1 = bi != bj || c + 1 >= h0 + r;
+            if (vec16 && keep0) {                 // n even: c + 1 < n as well; keep0 implies keep1
+                double2 v = __ldcg(reinterpret_cast<const double2*>(dst));
+                v.x -= acc[a][b][0];
+                v.y -= acc[a][b][1];
+                __stcg(reinterpret_cast<double2*>(dst), v);
+            } else {
+                if (keep0) __stcg(dst, __ldcg(dst) - acc[a][b][0]);
+                if (keep1 && j0 + c + 1 < n) __stcg(dst + 1, __ldcg(dst + 1) - acc[a][b][1]);
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kCholThreads, 1)
 chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned* bar, int32_t* status) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
-    double* rowbuf = opnd + 2 * 2 * kNB * kCholLd;                          // [2][64]
-    int* s_flag = reinterpret_cast<int*>(rowbuf + 2 * kNB);
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int* s_flag = reinterpret_cast<int*>(opnd + 2 * 2 * kNB * kCholLd);     // the strip panels alias opnd
+    const int tid = threadIdx.x;
     const int G = gridDim.x;
     const int nb = (n + kNB - 1) / kNB;
     unsigned epoch = 0;
@@ -153,35 +325,11 @@ chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned*
         const int k0 = k * kNB;
         // ------------------------------------------------------------------ strip phase
         const int panel_cols = n - k0 - kNB;                                // columns to the right of the block
-        const int groups = panel_cols > 0 ? (panel_cols + kCholPanelCols - 1) / kCholPanelCols : 0;
-        const int reps = groups > 0 ? groups : 1;                            // last block: diagonal only
+        const int chunks = panel_cols > 0 ? (panel_cols + kNB - 1) / kNB : 0;
+        const int reps = chunks > 0 ? chunks : 1;                            // last block: diagonal only
         for (int g = blockIdx.x; g < reps; g += G) {
-            // column owned by this thread: tid < 64 -> diagonal block column tid, else a panel column
-            const bool is_diag = tid < kNB;
-            const int gc = is_diag ? k0 + tid : k0 + kNB + g * kCholPanelCols + (tid - kNB);
-            const bool live = gc < n && (is_diag || groups > 0);
-            double col[kNB];
-#pragma unroll
-            for (int p = 0; p < kNB; ++p) {
-                double v = (is_diag && p == tid) ? 1.0 : 0.0;                // identity padding below n
-                if (live && k0 + p < n && (!is_diag || p <= tid)) v = __ldcg(A + (int64_t)(k0 + p) * ld + gc);
-                col[p] = v;
-            }
-            chol_strip_steps(col, rowbuf, is_diag, tid, g, k0, status, std::make_integer_sequence<int, kNB>());
-            if (live) {
-                if (is_diag) {
-                    if (g == 0) {
-#pragma unroll
-                        for (int p = 0; p < kNB; ++p)
-                            if (p <= tid && k0 + p < n) __stcg(A + (int64_t)(k0 + p) * ld + gc, col[p]);
-                    }
-                } else {
-#pragma unroll
-                    for (int p = 0; p < kNB; ++p)
-                        if (k0 + p < n) __stcg(A + (int64_t)(k0 + p) * ld + gc, col[p]);
-                }
-            }
-            __syncthreads();     // rowbuf is reused by the next repetition
+            chol_strip(A, ld, n, k0, chunks > 0 ? g : -1, g == 0, opnd, vec16, status);
+            __syncthreads();     // the panel buffers are reused by the next repetition and by the trailing phase
         }
         if (k == nb - 1) break;
         ++epoch;
@@ -190,68 +338,39 @@ chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned*
         // ------------------------------------------------------------------ trailing phase
         const int m = nb - 1 - k;
         const int T = m * (m + 1) / 2;
-        auto tile_ij = [&](int t, int& bi, int& bj) {
+        // tiles are cut into 64 / H row pieces so that a short tile list still spreads over the grid
+        const int H = 4 * T <= G ? 16 : (2 * T <= G ? 32 : 64);
+        const int pieces = kNB / H;
+        const int TP = T * pieces;
+        auto piece_coords = [&](int tp, int& bi, int& bj, int& h0) {
+            const int t = tp / pieces;
+            h0 = (tp - t * pieces) * H;
             int i = k + 1, rem = t;
             while (rem >= nb - i) { rem -= nb - i; ++i; }
             bi = i; bj = i + rem;
         };
+        auto load_piece = [&](int tp, int stg) {
+            int bi, bj, h0;
+            piece_coords(tp, bi, bj, h0);
+            double* dst = opnd + stg * 2 * kNB * kCholLd;
+            chol_load_block(dst, A, ld, n, k0, bi * kNB + h0, H, vec16);
+            chol_load_block(dst + kNB * kCholLd, A, ld, n, k0, bj * kNB, kNB, vec16);
+        };
         int stage = 0;
-        if ((int)blockIdx.x < T) {
-            int bi, bj;
-            tile_ij(blockIdx.x, bi, bj);
-            chol_load_block(opnd, A, ld, n, k0, bi * kNB, vec16);
-            chol_load_block(opnd + kNB * kCholLd, A, ld, n, k0, bj * kNB, vec16);
-        }
+        if ((int)blockIdx.x < TP) load_piece(blockIdx.x, 0);
         cp_async_commit();
-        for (int t = blockIdx.x; t < T; t += G) {
-            int bi, bj;
-            tile_ij(t, bi, bj);
-            if (t + G < T) {
-                int ni, nj;
-                tile_ij(t + G, ni, nj);
-                double* nxt = opnd + (stage ^ 1) * 2 * kNB * kCholLd;
-                chol_load_block(nxt, A, ld, n, k0, ni * kNB, vec16);
-                chol_load_block(nxt + kNB * kCholLd, A, ld, n, k0, nj * kNB, vec16);
-            }
+        for (int tp = blockIdx.x; tp < TP; tp += G) {
+            if (tp + G < TP) load_piece(tp + G, stage ^ 1);
             cp_async_commit();
             cp_async_wait<1>();
             __syncthreads();
-            const double* as = opnd + stage * 2 * kNB * kCholLd;            // as[kk][m] = U[k0 + kk][i0 + m]
-            const double* bs = as + kNB * kCholLd;                           // bs[kk][n] = U[k0 + kk][j0 + n]
-            const int wm0 = (warp >> 2) * 32, wn0 = (warp & 3) * 16;
-            const int lq = lane >> 2, lr = lane & 3;
-            double acc[4][2][2];
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
-#pragma unroll 4
-            for (int kk = 0; kk < kNB; kk += 4) {
-                double af[4], bf[2];
-#pragma unroll
-                for (int a = 0; a < 4; ++a) af[a] = as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
-#pragma unroll
-                for (int b = 0; b < 2; ++b) bf[b] = bs[(kk + lr) * kCholLd + wn0 + b * 8 + lq];
-#pragma unroll
-                for (int a = 0; a < 4; ++a)
-#pragma unroll
-                    for (int b = 0; b < 2; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
-            }
-            const int i0 = bi * kNB, j0 = bj * kNB;
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-                const int r = wm0 + a * 8 + lq;
-#pragma unroll
-                for (int b = 0; b < 2; ++b)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int c = wn0 + b * 8 + 2 * lr + e;
-                        if (i0 + r < n && j0 + c < n && (bi != bj || c >= r)) {
-                            double* dst = A + (int64_t)(i0 + r) * ld + j0 + c;
-                            __stcg(dst, __ldcg(dst) - acc[a][b][e]);
-                        }
-                    }
-            }
+            int bi, bj, h0;
+            piece_coords(tp, bi, bj, h0);
+            const double* as = opnd + stage * 2 * kNB * kCholLd;            // as[kk][m] = U[k0 + kk][i0 + h0 + m]
+            const double* bs = as + kNB * kCholLd;                           // bs[kk][c] = U[k0 + kk][j0 + c]
+            if (H == 64) chol_trailing_piece<64>(A, ld, n, as, bs, bi, bj, h0, vec16);
+            else if (H == 32) chol_trailing_piece<32>(A, ld, n, as, bs, bi, bj, h0, vec16);
+            else chol_trailing_piece<16>(A, ld, n, as, bs, bi, bj, h0, vec16);
             __syncthreads();     // all warps are done with this stage before it is refilled
             stage ^= 1;
         }
