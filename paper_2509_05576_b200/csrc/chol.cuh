@@ -118,17 +118,15 @@ __device__ __forceinline__ void chol_load_block(double* dst, const double* __res
 // MMA accumulator fragments (warp w owns strip columns 16 w .. 16 w + 15, all 64 rows).  Pivots are taken eight
 // at a time.  For pivot block b:
 //   1. every warp publishes its piece of rows 8 b .. 8 b + 7 (the row panel R) to shared memory;
-//   2. every warp factorises the 8 x 8 diagonal mini-block M = U_M^T U_M redundantly, one column per lane with
-//      warp shuffles, and carries the identity along to obtain W = U_M^-T;
+//   2. four warps factorise the 8 x 8 diagonal mini-block M = U_M^T U_M (redundantly, all of M in every lane)
+//      and carry the identity along to obtain W = U_M^-T;
 //   3. the new rows U[8 b .. 8 b + 7][:] = W R come from two MMAs per fragment;
 //   4. they are published and subtracted from the rows below, A[i][c] -= U[p][i] U[p][c], again by MMA.
-// Two block-wide barriers per eight pivots; the only serial chain is the eight reciprocal square roots of step 2.
+// Three block-wide barriers per eight pivots; the only serial chain is the eight reciprocal square roots of step 2.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kStripLd = 132;                                            // row stride of the 8-row panels
 constexpr int kStripSmemDoubles = 2 * 8 * kStripLd + (kCholThreads / 32) * 64;
 static_assert(kStripSmemDoubles <= 2 * 2 * kNB * kCholLd, "the strip panels alias the trailing-phase operand buffers");
-
-__device__ __forceinline__ double shfl_f64(double x, int src) { return __shfl_sync(0xffffffffu, x, src); }
 
 template <int B>
 __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
@@ -141,32 +139,44 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
         *reinterpret_cast<double2*>(Rbuf + lq * kStripLd + c0 + 8 * cb + 2 * lr) =
             make_double2(acc[B][cb][0], acc[B][cb][1]);
     __syncthreads();
-    // 2. mini-block factorisation: lanes 0..7 own the columns of M, lanes 8..15 the columns of the identity
-    const int jj = lane & 15;
-    double v[8];
+    // 2. warps 0..3 (one per scheduler) each factorise M; every lane holds all of M, so the serial chain of
+    //    eight reciprocal square roots has no data exchange in it.  Lane j carries column j of the identity along,
+    //    which becomes column j of W = U_M^-T.
+    if (warp < 4) {
+        double m[8][8];
 #pragma unroll
-    for (int p = 0; p < 8; ++p)
-        v[p] = jj < 8 ? Rbuf[p * kStripLd + 8 * B + jj] : (p == jj - 8 ? 1.0 : 0.0);
+        for (int p = 0; p < 8; ++p)
 #pragma unroll
-    for (int p = 0; p < 8; ++p) {
-        const double x = v[p];
-        double d = shfl_f64(x, p);
-        if (!(d > 0.0) || !isfinite(d)) {
-            if (reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + p);
-            d = 1.0;
+            for (int j = p; j < 8; ++j) m[p][j] = Rbuf[p * kStripLd + 8 * B + j];
+        const int jc = lane & 7;
+        double x[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = i == jc ? 1.0 : 0.0;
+#pragma unroll
+        for (int p = 0; p < 8; ++p) {
+            double d = m[p][p];
+            const bool ok = d > 0.0 && isfinite(d);
+            if (!ok && reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + p);
+            d = ok ? d : 1.0;
+            const double rs = rsqrt(d);
+            const double inv = rs * rs;
+            const double tx = x[p] * inv;
+            x[p] *= rs;
+#pragma unroll
+            for (int i = p + 1; i < 8; ++i) {
+                const double f = m[p][i] * inv;
+                x[i] = fma(-m[p][i], tx, x[i]);
+#pragma unroll
+                for (int j = i; j < 8; ++j) m[i][j] = fma(-f, m[p][j], m[i][j]);
+            }
         }
-        const double rs = rsqrt(d);
-        const double t = x * (rs * rs);
-        v[p] = x * rs;
+        if (lane < 8) {
 #pragma unroll
-        for (int i = p + 1; i < 8; ++i) v[i] = fma(-shfl_f64(x, i), t, v[i]);
+            for (int p = 0; p < 8; ++p) Wbuf[warp * 64 + p * 8 + lane] = x[p];    // W[p][j] = (U_M^-T)[p][j]
+        }
     }
-    double* wb = Wbuf + warp * 64;
-    if (lane >= 8 && lane < 16) {
-#pragma unroll
-        for (int p = 0; p < 8; ++p) wb[p * 8 + (lane - 8)] = v[p];      // W[p][j] = (U_M^-T)[p][j]
-    }
-    __syncwarp();
+    __syncthreads();
+    const double* wb = Wbuf + (warp & 3) * 64;
     // 3. new rows = W R
     const double a0 = wb[lq * 8 + lr], a1 = wb[lq * 8 + 4 + lr];
 #pragma unroll
@@ -271,16 +281,35 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ A, int6
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int wm0 = (warp >> 2) * (H / 2), wn0 = (warp & 3) * 16;
     const int lq = lane >> 2, lr = lane & 3;
+    const int i0 = bi * kNB + h0, j0 = bj * kNB;
+    // the old values of the tile are fetched first, so that their latency hides behind the MMAs
     double acc[FM][2][2];
+    bool keep[FM][2][2];
 #pragma unroll
-    for (int a = 0; a < FM; ++a)
+    for (int a = 0; a < FM; ++a) {
+        const int r = wm0 + a * 8 + lq;
 #pragma unroll
-        for (int b = 0; b < 2; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
+        for (int b = 0; b < 2; ++b) {
+            const int c = wn0 + b * 8 + 2 * lr;
+            const bool in = i0 + r < n && j0 + c < n;
+            keep[a][b][0] = in && (bi != bj || c >= h0 + r);
+            keep[a][b][1] = in && j0 + c + 1 < n && (bi != bj || c + 1 >= h0 + r);
+            const double* src = A + (int64_t)(i0 + r) * ld + j0 + c;
+            if (vec16 && keep[a][b][0]) {             // n even: the pair is inside; keep[0] implies keep[1]
+                const double2 v = __ldcg(reinterpret_cast<const double2*>(src));
+                acc[a][b][0] = v.x;
+                acc[a][b][1] = v.y;
+            } else {
+                acc[a][b][0] = keep[a][b][0] ? __ldcg(src) : 0.0;
+                acc[a][b][1] = keep[a][b][1] ? __ldcg(src + 1) : 0.0;
+            }
+        }
+    }
 #pragma unroll 4
     for (int kk = 0; kk < kNB; kk += 4) {
         double af[FM], bf[2];
 #pragma unroll
-        for (int a = 0; a < FM; ++a) af[a] = as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
+        for (int a = 0; a < FM; ++a) af[a] = -as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
 #pragma unroll
         for (int b = 0; b < 2; ++b) bf[b] = bs[(kk + lr) * kCholLd + wn0 + b * 8 + lq];
 #pragma unroll
@@ -288,24 +317,18 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ A, int6
 #pragma unroll
             for (int b = 0; b < 2; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
     }
-    const int i0 = bi * kNB + h0, j0 = bj * kNB;
 #pragma unroll
     for (int a = 0; a < FM; ++a) {
         const int r = wm0 + a * 8 + lq;
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
             const int c = wn0 + b * 8 + 2 * lr;
-            if (i0 + r >= n || j0 + c >= n) continue;
             double* dst = A + (int64_t)(i0 + r) * ld + j0 + c;
-            const bool keep0 = bi != bj || c >= h0 + r, keep1 = bi != bj || c + 1 >= h0 + r;
-            if (vec16 && keep0) {                 // n even: c + 1 < n as well; keep0 implies keep1
-                double2 v = __ldcg(reinterpret_cast<const double2*>(dst));
-                v.x -= acc[a][b][0];
-                v.y -= acc[a][b][1];
-                __stcg(reinterpret_cast<double2*>(dst), v);
+            if (vec16 && keep[a][b][0]) {
+                __stcg(reinterpret_cast<double2*>(dst), make_double2(acc[a][b][0], acc[a][b][1]));
             } else {
-                if (keep0) __stcg(dst, __ldcg(dst) - acc[a][b][0]);
-                if (keep1 && j0 + c + 1 < n) __stcg(dst + 1, __ldcg(dst + 1) - acc[a][b][1]);
+                if (keep[a][b][0]) __stcg(dst, acc[a][b][0]);
+                if (keep[a][b][1]) __stcg(dst + 1, acc[a][b][1]);
             }
         }
     }
