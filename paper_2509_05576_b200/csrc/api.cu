@@ -142,6 +142,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(c * sizeof(int32_t));                       // inverse permutation
             add(loss_partials_count(rows, cols) * sizeof(double));
             add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
+            add(((size_t)cdiv(rows, kSweepRows) + 1) * sizeof(unsigned));   // per-row-group progress counters of the sweep
             break;
         default:
             return 0;
@@ -269,11 +270,6 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
         return PTQ_ERR_INVALID_ARG;
     if (!aligned16(Hinv) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(colloop_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kColloopSmem);
-        attr_done = true;
-    }
     const int n = cols;
     Carver cv(ws);
     double* U = cv.take<double>((size_t)n * n);
@@ -284,6 +280,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     int32_t* invperm = cv.take<int32_t>(n);
     double* partials = cv.take<double>(loss_partials_count(rows, cols));
     unsigned* bar = cv.take<unsigned>(2);
+    unsigned* sweep_flags = cv.take<unsigned>((size_t)cdiv(rows, kSweepRows) + 1);
 
     // flags and invperm are adjacent pieces of the workspace: clear both
     if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
@@ -295,25 +292,8 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     int st = cholesky_upper(U, n, bar, status, stream);   // blocked Eq. 12
     if (st) return st;
 
-    const int row_ctas = cdiv(rows, kRowsPerCta);
-    for (int p0 = 0; p0 < n; p0 += kNB) {
-        const int kb = n - p0 < kNB ? n - p0 : kNB;
-        {
-            Launch l(K_COLLOOP_BLOCK, stream);
-            colloop_block_kernel<<<row_ctas, 128, kColloopSmem, stream>>>(Wp, rows, n, p0, kb, U, scale, zero, bits, E,
-                                                                          codes_p);
-        }
-        const int rest = n - p0 - kb;
-        if (rest <= 0) break;
-        GemmParams g = gemm_defaults();     // deferred Eq. 11: W[:, later] -= E[:, block] U[block, later]
-        g.A = E + p0; g.lda = n; g.a_trans = 0;
-        g.B = U + (int64_t)p0 * n + p0 + kb; g.ldb = n; g.b_trans = 0;
-        g.C = Wp + p0 + kb; g.ldc = n;
-        g.M = rows; g.N = rest; g.K = kb;
-        g.alpha = -1.0; g.beta = 1.0;
-        st = launch_dgemm(K_DGEMM_WUPDATE, g, 1, stream);
-        if (st) return st;
-    }
+    st = sweep_launch(Wp, U, E, codes_p, scale, zero, rows, n, bits, sweep_flags, status, stream);
+    if (st) return st;
 
     const bool want_loss = H_undamped && loss_out;
     double* dW = want_loss ? Wp : nullptr;
