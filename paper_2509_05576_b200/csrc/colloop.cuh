@@ -3,8 +3,7 @@
 // With A the permuted inverse Hessian and A = U^T U its upper Cholesky factor, the matrix that Eq. 12 leaves
 // before step p has row p equal to sqrt(pivot) * U[p, p:], so Eq. 11 for column p reads
 //     e_i = (w_ip - q_ip) / U[p][p],      w_ij -= e_i * U[p][j]   for j > p.
-// Columns are processed in blocks of 64: inside a block every row is swept by one thread that keeps the
-// block's 64 weights in registers; the effect of the block on a later block is one float64 MMA tile,
+// Columns are processed in blocks of 64; the effect of a block on a later block is one float64 MMA tile,
 // W[:, later] -= E[:, block] U[block, later].
 #pragma once
 #include "common.cuh"
@@ -51,23 +50,31 @@ __global__ void gather_w_kernel(const float* __restrict__ W, int rows, int cols,
 // Rows never interact (Sec. 4.2 step 4: every row of the current column is quantized at once, independently), so
 // the rows are cut into groups of 32 and each group is an independent pipeline.  A group is served by `cpg` CTAs;
 // the 64-column blocks are dealt to them round-robin (CTA i owns blocks i, i + cpg, ...).  The owner of block b
-//   - quantizes it: one warp, one row per lane, the block's 64 weights in float64 registers, the 64 x 64 diagonal
-//     block of U in shared memory: c = clamp(rint(w / s) + z), e = (w - q) / U_pp, w_j -= e U_pj (Eq. 11 inside the
-//     block), and writes the scaled errors E[:, b] and the codes;
-//   - raises the group's counter to b + 1.
-// Every CTA of the group then applies E[:, b] to the blocks IT owns: W[:, b'] -= E[:, b] U[b, b'] (the deferred part
-// of Eq. 11), a 32 x 64 x 64 float64 tensor-core MMA tile per block.  All updates of one block are made by its owner,
-// in order, so no block is ever touched by two CTAs; the only cross-CTA dependency is "E[:, b] is ready".  The owner of
-// block b + 1 updates that block first and starts quantizing at once; its other blocks catch up afterwards.
+// quantizes it, writes the scaled errors E[:, b] and the codes, and raises the group's counter to b + 1.  Every CTA
+// of the group then applies E[:, b] to the blocks IT owns: W[:, b'] -= E[:, b] U[b, b'] (the deferred part of Eq. 11),
+// a 32 x 64 x 64 float64 tensor-core MMA tile per block.  All updates of one block are made by its owner, in order, so
+// no block is ever touched by two CTAs; the only cross-CTA dependency is "E[:, b] is ready".  The owner of block b + 1
+// updates that block first, straight into registers, and starts quantizing at once; its other blocks catch up later.
 // Waits on the counter are bounded; when one expires the CTA raises the abort word, reports PTQ_ERR_TIMEOUT and leaves.
+//
+// Inside a block the 32 x 64 tile of W lives in registers as 8 x 8 MMA accumulator fragments, warp k holding columns
+// 8 k .. 8 k + 7 of all 32 rows.  Columns are quantized eight at a time ("mini-block" m, owned by warp m):
+//   - warp m turns its fragments into one-row-per-lane form and runs the eight dependent steps
+//         c = clamp(rint(w / s) + z),  d = w - q,  w_j -= d U[p][j] / U[p][p]   (j inside the mini-block),
+//     with warp-private shared-memory staging only, then publishes the 32 x 8 differences d;
+//   - the warps to its right subtract d (U[p][j] / U[p][p]) from their fragments: a rank-8 update, two MMAs per
+//     fragment.  One block-wide barrier per mini-block.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kSweepThreads = 256;
 constexpr int kSweepRows = 32;
 constexpr int kSweepLd = kNB + 4;                                   // 68: conflict-free MMA operand stride
-constexpr int kSweepWsLd = kNB + 1;                                 // 65: conflict-free row-per-lane access
-constexpr size_t kSweepSmemBytes =
-    sizeof(double) * (kNB * kNB + kSweepRows * kSweepWsLd + kNB + kSweepRows * kSweepLd + 2 * kNB * kSweepLd) +
-    kSweepRows * (kNB + 4) + 16;
+constexpr int kSweepEsLd = kNB + 1;                                 // 65: row-per-lane writes of E
+constexpr int kSweepTLd = 9;                                        // fragment <-> row-per-lane staging
+constexpr int kSweepDLd = 12;                                       // 32 x 8 differences as MMA operand A
+constexpr int kSweepSmemDoubles = kNB * kSweepLd /*Us*/ + kNB /*rdiag*/ + kSweepRows * kSweepEsLd /*Es*/ +
+                                  kSweepRows * kSweepTLd /*T*/ + 2 * kSweepRows * kSweepDLd /*Dm*/ +
+                                  kSweepRows * kSweepLd /*Ea*/ + 2 * kNB * kSweepLd /*Bb*/;
+constexpr size_t kSweepSmemBytes = sizeof(double) * kSweepSmemDoubles + kSweepRows * (kNB + 4) + 16;
 
 struct SweepParams {
     double* Wp;             // [rows x n] permuted weights, float64, updated in place
@@ -80,20 +87,6 @@ struct SweepParams {
     unsigned* flags;        // [groups] finished blocks per group, then [1] abort word; zero at launch
     int32_t* status;
 };
-
-// quant(): the nearest level of the row's grid (ties to even) of w, clamped to the code range.  w / s is a true
-// float64 division by definition; the product w * (1 / s) differs from it by less than 4e-16 |w / s|, so whenever that
-// product is further than 1e-6 from a rounding boundary (and below 1e9 in magnitude) both round to the same integer and
-// the division is skipped.
-__device__ __forceinline__ double quant_code_fast(double w, double sc, double rsc, double zp, double maxq) {
-    double v = w * rsc;
-    double rv = rint(v);
-    if (!(fabs(v - rv) < 0.5 - 1e-6) || !(fabs(v) < 1e9)) rv = rint(w / sc);
-    double c = rv + zp;
-    c = fmax(c, 0.0);
-    c = fmin(c, maxq);
-    return c;
-}
 
 // Copies a tile of nr x nc doubles (nc even when vec16) from src (row stride ld) into dst (row stride dst_ld);
 // rows at or beyond rmax and columns at or beyond cmax are filled with zeros.
@@ -115,29 +108,52 @@ __device__ __forceinline__ void sweep_load_tile(double* dst, int dst_ld, const d
     }
 }
 
-template <int... Ps>
-__device__ __forceinline__ void sweep_chain_steps(double (&w)[kNB], const double* Us, const double* rdiag, double* ws_row,
-                                                  uint8_t* cs_row, double sc, double rsc, double zp, double maxq,
-                                                  std::integer_sequence<int, Ps...>) {
-    auto step = [&](auto pc) {
-        constexpr int P = decltype(pc)::value;
-        const double c = quant_code_fast(w[P], sc, rsc, zp, maxq);
-        const double q = sc * (c - zp);
-        const double e = (w[P] - q) * rdiag[P];
+// Per-row constants of the quantizer: scale, 1 / scale, zero-point and the clamp range [-z, maxq - z] of rint(w / s)
+// (clamping that integer is the same as clamping the code to [0, maxq], because the zero-point is an integer).
+struct RowGrid {
+    double sc, rsc, zp, lo, hi;
+};
+
+// Eight dependent quantization steps of one row (one lane) on the mini-block whose weights are v[0..7].
+// us points at U'[8 m][8 m] (rows of U divided by their pivots, row stride kSweepLd).  Returns the differences
+// d_p = w_p - q_p in v[] and the clamped level indices in lev[].
+//
+// EXACT = false: the level index rint(w / s) -- by definition a true float64 division -- is taken from the product
+// w * (1 / s), which differs from the quotient by less than 4e-16 |w / s|; whenever the product is further than 1e-6
+// from a rounding boundary (and below 1e9 in magnitude) both round to the same integer.  The return value tells whether
+// some step was closer than that, in which case the caller repeats the mini-block with EXACT = true (the division).
+// Rounding: (v + 1.5 * 2^52) - 1.5 * 2^52 is round-to-nearest-even for |v| < 2^51.
+template <bool EXACT>
+__device__ __forceinline__ bool sweep_chain8(double (&v)[8], double (&lev)[8], const double* us, const RowGrid& g) {
+    bool danger = false;
 #pragma unroll
-        for (int j = P + 1; j < kNB; ++j) w[j] = fma(-e, Us[P * kNB + j], w[j]);
-        ws_row[P] = e;
-        cs_row[P] = (uint8_t)(int)c;
-    };
-    (step(std::integral_constant<int, Ps>()), ...);
+    for (int p = 0; p < 8; ++p) {
+        double rv;
+        if (EXACT) {
+            rv = rint(v[p] / g.sc);
+        } else {
+            const double t = v[p] * g.rsc;
+            rv = (t + 6755399441055744.0) - 6755399441055744.0;
+            danger |= !(fabs(t - rv) < 0.5 - 1e-6) || !(fabs(t) < 1e9);
+        }
+        const double rvc = fmin(fmax(rv, g.lo), g.hi);
+        const double d = v[p] - g.sc * rvc;
+#pragma unroll
+        for (int j = p + 1; j < 8; ++j) v[j] = fma(-d, us[p * kSweepLd + j], v[j]);
+        v[p] = d;
+        lev[p] = rvc;
+    }
+    return danger;
 }
 
 __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParams prm) {
     extern __shared__ __align__(16) unsigned char sweep_smem[];
-    double* Us = reinterpret_cast<double*>(sweep_smem);                // [64][64] diagonal block of U
-    double* Ws = Us + kNB * kNB;                                       // [32][65] block of W, later of E
-    double* rdiag = Ws + kSweepRows * kSweepWsLd;                      // [64]
-    double* Ea = rdiag + kNB;                                          // [32][68] MMA operand A: E[:, e]
+    double* Us = reinterpret_cast<double*>(sweep_smem);                // [64][68] diagonal block of U, rows / pivot
+    double* rdiag = Us + kNB * kSweepLd;                               // [64] 1 / U_pp
+    double* Es = rdiag + kNB;                                          // [32][65] scaled errors of the block
+    double* T = Es + kSweepRows * kSweepEsLd;                          // [32][9] staging of the current mini-block
+    double* Dm = T + kSweepRows * kSweepTLd;                           // [2][32][12] differences of a mini-block
+    double* Ea = Dm + 2 * kSweepRows * kSweepDLd;                      // [32][68] MMA operand A: E[:, e]
     double* Bb = Ea + kSweepRows * kSweepLd;                           // [2][64][68] MMA operand B: U[e, b']
     uint8_t* Cs = reinterpret_cast<uint8_t*>(Bb + 2 * kNB * kSweepLd); // [32][68] codes of the block
     int* s_flag = reinterpret_cast<int*>(Cs + kSweepRows * (kNB + 4));
@@ -149,61 +165,122 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
     const int G = gridDim.x;
     unsigned* abort_word = prm.flags + groups;
     const double maxq = (double)((1 << prm.bits) - 1);
+    const int lq = lane >> 2, lr = lane & 3;
+    // far-update MMA tile coordinates: 8 warps as 2 x 4, each 16 x 16
+    const int wm0 = (warp >> 2) * 16, wn0 = (warp & 3) * 16;
 
     int cpg = 1, g_first = blockIdx.x, g_step = G, ci = 0;
     if (groups < G) {
-        cpg = G / groups;
-        if (cpg > nb) cpg = nb;
         const int per = G / groups;                // CTAs reserved per group; only the first cpg of them work
+        cpg = per < nb ? per : nb;
         g_first = blockIdx.x / per;
         ci = blockIdx.x - g_first * per;
         g_step = groups;                           // one group per CTA
         if (g_first >= groups || ci >= cpg) return;
     }
 
+    // diagonal block of U for block b: Us = rows divided by their pivots, rdiag = 1 / pivot
+    auto load_diag = [&](int b) {
+        const int p0 = b * kNB;
+        const int kb = n - p0 < kNB ? n - p0 : kNB;
+        for (int idx = tid; idx < kNB * kNB; idx += kSweepThreads) {
+            const int r = idx >> 6, c = idx & 63;
+            double v = (r == c) ? 1.0 : 0.0;
+            if (r < kb && c < kb && c >= r) v = __ldcg(prm.U + (int64_t)(p0 + r) * n + p0 + c);
+            Us[r * kSweepLd + c] = v;
+        }
+        __syncthreads();
+        if (tid < kNB) rdiag[tid] = 1.0 / Us[tid * kSweepLd + tid];
+        __syncthreads();
+        for (int idx = tid; idx < kNB * kNB; idx += kSweepThreads) Us[(idx >> 6) * kSweepLd + (idx & 63)] *= rdiag[idx >> 6];
+    };
+
     for (int g = g_first; g < groups; g += g_step) {
         const int r0 = g * kSweepRows;
         int lazy = 0;
+        bool prepared = false;           // Us / rdiag / blk already hold the block about to be quantized
+        // the block being quantized: fragment a = rows 8 a + lq, columns 8 warp + 2 lr + {0, 1}
+        double blk[4][2];
         for (int b = 0; b < nb; ++b) {
             const int p0 = b * kNB;
             const int kb = n - p0 < kNB ? n - p0 : kNB;
             const bool mine = (b % cpg) == ci;
+            const bool next_mine = cpg > 1 && b + 1 < nb && ((b + 1) % cpg) == ci;
+            if (next_mine) {
+                // block b + 1 is quantized here next: what does not depend on E[:, b] is fetched before waiting for it
+                __syncthreads();
+                sweep_load_tile(Bb, kSweepLd, prm.U, n, p0, p0 + kNB, kNB, kNB, n, n, prm.vec16);
+                cp_async_commit();
+                load_diag(b + 1);
+            }
             if (mine) {
                 // ------------------------------------------------------------ quantize block b
-                for (int idx = tid; idx < kNB * kNB; idx += kSweepThreads) {
-                    const int r = idx >> 6, c = idx & 63;
-                    double v = (r == c) ? 1.0 : 0.0;
-                    if (r < kb && c < kb && c >= r) v = __ldcg(prm.U + (int64_t)(p0 + r) * n + p0 + c);
-                    Us[idx] = v;
-                }
-                for (int idx = tid; idx < kSweepRows * kNB; idx += kSweepThreads) {
-                    const int r = idx >> 6, c = idx & 63;
-                    double v = 0.0;
-                    if (r0 + r < rows && c < kb) v = __ldcg(prm.Wp + (int64_t)(r0 + r) * n + p0 + c);
-                    Ws[r * kSweepWsLd + c] = v;
-                }
-                __syncthreads();
-                if (tid < kNB) rdiag[tid] = 1.0 / Us[tid * kNB + tid];
-                __syncthreads();
-                if (warp == 0) {
-                    const int row = r0 + lane;
-                    const bool live = row < rows;
-                    const double sc = live ? (double)prm.scale[row] : 1.0;
-                    const double zp = live ? (double)prm.zero[row] : 0.0;
-                    const double rsc = 1.0 / sc;
-                    double w[kNB];
+                if (!prepared) {
+                    __syncthreads();
+                    load_diag(b);
 #pragma unroll
-                    for (int c = 0; c < kNB; ++c) w[c] = Ws[lane * kSweepWsLd + c];
-                    sweep_chain_steps(w, Us, rdiag, Ws + lane * kSweepWsLd, Cs + lane * (kNB + 4), sc, rsc, zp, maxq,
-                                      std::make_integer_sequence<int, kNB>());
+                    for (int a = 0; a < 4; ++a)
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int r = r0 + 8 * a + lq, c = p0 + 8 * warp + 2 * lr + e;
+                            blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
+                        }
+                }
+                __syncthreads();
+                const int row = r0 + lane;
+                const bool live = row < rows;
+                RowGrid rg;
+                rg.sc = live ? (double)prm.scale[row] : 1.0;
+                rg.zp = live ? (double)prm.zero[row] : 0.0;
+                rg.rsc = 1.0 / rg.sc;
+                rg.lo = -rg.zp;
+                rg.hi = maxq - rg.zp;
+#pragma unroll
+                for (int m = 0; m < 8; ++m) {
+                    double* dm = Dm + (m & 1) * kSweepRows * kSweepDLd;
+                    if (warp == m) {
+                        // fragments -> one row per lane
+#pragma unroll
+                        for (int a = 0; a < 4; ++a)
+#pragma unroll
+                            for (int e = 0; e < 2; ++e) T[(8 * a + lq) * kSweepTLd + 2 * lr + e] = blk[a][e];
+                        __syncwarp();
+                        double v[8], lev[8];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) v[c] = T[lane * kSweepTLd + c];
+                        const double* us = Us + (8 * m) * kSweepLd + 8 * m;
+                        const bool danger = sweep_chain8<false>(v, lev, us, rg);
+                        if (__any_sync(0xffffffffu, danger)) {
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) v[c] = T[lane * kSweepTLd + c];
+                            sweep_chain8<true>(v, lev, us, rg);
+                        }
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            dm[lane * kSweepDLd + c] = v[c];
+                            Es[lane * kSweepEsLd + 8 * m + c] = v[c] * rdiag[8 * m + c];
+                            Cs[lane * (kNB + 4) + 8 * m + c] = (uint8_t)(int)(lev[c] + rg.zp);
+                        }
+                    }
+                    if (m == 7) break;
+                    __syncthreads();
+                    if (warp > m) {
+                        // rank-8 update of this warp's columns: blk -= d (U'[8 m .. 8 m + 7][8 warp .. 8 warp + 7])
+                        const double b0 = Us[(8 * m + lr) * kSweepLd + 8 * warp + lq];
+                        const double b1 = Us[(8 * m + 4 + lr) * kSweepLd + 8 * warp + lq];
+#pragma unroll
+                        for (int a = 0; a < 4; ++a) {
+                            const double a0 = -dm[(8 * a + lq) * kSweepDLd + lr];
+                            const double a1 = -dm[(8 * a + lq) * kSweepDLd + 4 + lr];
+                            dmma_884(blk[a][0], blk[a][1], a0, b0);
+                            dmma_884(blk[a][0], blk[a][1], a1, b1);
+                        }
+                    }
                 }
                 __syncthreads();
                 for (int idx = tid; idx < kSweepRows * kNB; idx += kSweepThreads) {
                     const int r = idx >> 6, c = idx & 63;
-                    if (r0 + r < rows && c < kb) {
-                        __stcg(prm.E + (int64_t)(r0 + r) * n + p0 + c, Ws[r * kSweepWsLd + c]);
-                        prm.codes_p[(int64_t)(r0 + r) * n + p0 + c] = Cs[r * (kNB + 4) + c];
-                    }
+                    if (r0 + r < rows && c < kb) __stcg(prm.E + (int64_t)(r0 + r) * n + p0 + c, Es[r * kSweepEsLd + c]);
                 }
                 if (cpg > 1) {
                     __syncthreads();
@@ -212,6 +289,11 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         atomicExch(&prm.flags[g], (unsigned)(b + 1));
                     }
                 }
+                for (int idx = tid; idx < kSweepRows * kNB; idx += kSweepThreads) {
+                    const int r = idx >> 6, c = idx & 63;
+                    if (r0 + r < rows && c < kb) prm.codes_p[(int64_t)(r0 + r) * n + p0 + c] = Cs[r * (kNB + 4) + c];
+                }
+                prepared = false;
             } else {
                 // ------------------------------------------------------------ wait for E[:, b]
                 if (tid == 0) {
@@ -229,29 +311,42 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                 }
                 __syncthreads();
                 if (*s_flag == 0) {
+                    cp_async_wait<0>();
                     if (tid == 0) report(prm.status, PTQ_ERR_TIMEOUT, blockIdx.x, 2);
                     return;
                 }
             }
             if (b + 1 >= nb) break;
             // ---------------------------------------------------------------- deferred Eq. 11 on the owned blocks
-            const bool next_mine = cpg > 1 && ((b + 1) % cpg) == ci;
-            int e_lo, b_first, b_last;
             if (next_mine) {
-                e_lo = b; b_first = b + 1; b_last = b + 1;                 // only the block about to be quantized
-            } else {
-                e_lo = lazy;
-                b_first = b + 1 + (((ci - (b + 1)) % cpg) + cpg) % cpg;     // first owned block beyond b
-                b_last = nb - 1;
-                lazy = b + 1;
-            }
-            if (b_first > b_last) {
-                // nothing owned beyond b: this CTA is finished with the group once nothing is deferred either
-                bool later = false;
-                for (int bb = b + 1; bb < nb; ++bb) later |= (bb % cpg) == ci;
-                if (!later) break;
+                // block b + 1 only, straight into the fragments the chain starts from; the other blocks catch up later
+                sweep_load_tile(Ea, kSweepLd, prm.E, n, r0, p0, kSweepRows, kNB, rows, n, prm.vec16);
+                cp_async_commit();
+#pragma unroll
+                for (int a = 0; a < 4; ++a)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const int r = r0 + 8 * a + lq, c = p0 + kNB + 8 * warp + 2 * lr + e;
+                        blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
+                    }
+                cp_async_wait<0>();
+                __syncthreads();
+#pragma unroll 4
+                for (int kk = 0; kk < kNB; kk += 4) {
+                    const double bf = Bb[(kk + lr) * kSweepLd + 8 * warp + lq];
+#pragma unroll
+                    for (int a = 0; a < 4; ++a) {
+                        const double af = -Ea[(8 * a + lq) * kSweepLd + kk + lr];
+                        dmma_884(blk[a][0], blk[a][1], af, bf);
+                    }
+                }
+                prepared = true;
                 continue;
             }
+            const int b_first = b + 1 + (((ci - (b + 1)) % cpg) + cpg) % cpg;     // first owned block beyond b
+            if (b_first >= nb) break;                                               // nothing left for this CTA
+            const int e_lo = lazy;
+            lazy = b + 1;
             for (int e = e_lo; e <= b; ++e) {
                 // operand A: E[r0 .. r0+31][64 e .. 64 e + 63]
                 __syncthreads();
@@ -259,14 +354,12 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                 int stage = 0;
                 sweep_load_tile(Bb, kSweepLd, prm.U, n, e * kNB, b_first * kNB, kNB, kNB, n, n, prm.vec16);
                 cp_async_commit();
-                for (int bp = b_first; bp <= b_last; bp += cpg) {
-                    if (bp + cpg <= b_last)
+                for (int bp = b_first; bp < nb; bp += cpg) {
+                    if (bp + cpg < nb)
                         sweep_load_tile(Bb + (stage ^ 1) * kNB * kSweepLd, kSweepLd, prm.U, n, e * kNB,
                                         (bp + cpg) * kNB, kNB, kNB, n, n, prm.vec16);
                     cp_async_commit();
                     // old values of the tile first (their latency hides behind the MMAs)
-                    const int wm0 = (warp >> 2) * 16, wn0 = (warp & 3) * 16;
-                    const int lq = lane >> 2, lr = lane & 3;
                     const int j0 = bp * kNB;
                     double acc[2][2][2];
                     bool keep[2][2][2];
@@ -324,7 +417,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                 }
                 cp_async_wait<0>();
             }
-            __syncthreads();             // the updated block is read back through global memory by the next chain
+            __syncthreads();             // the updated blocks are read back through global memory later
         }
     }
 }
