@@ -1,0 +1,103 @@
+"""GPU parity on layers taken from the benchmark configurations (ResNet-50-shaped, YOLOv5s-shaped and the square /
+wide scaling shapes), at their full sizes, through the C-ABI, against the CPU oracle on the same seeded inputs.
+
+The oracle applies Eq. 12 literally, which costs cols^3 / 3 multiply-adds per layer whatever the number of rows; for
+the widest layers it therefore sweeps a seeded subset of rows only (rows are independent once the column order and
+the inverse Hessian are fixed, Sec. 4.2 step 4), while Hessian, inverse, scores and order are compared in full.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2509_05576_b200 import ptq
+from paper_2509_05576_b200 import workloads as wl
+from parity import assert_layer_parity, compare_codes, gpu_layer, oracle_layer, LOSS_RTOL, WHAT_RTOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _find(specs, key):
+    for s in specs:
+        if key in s.name:
+            return s
+    raise KeyError(key)
+
+
+def _full(spec):
+    W, X = wl.make_layer(spec)
+    ref = oracle_layer(W, X, spec.bits, spec.damp)
+    g = gpu_layer(W, X, spec.bits, spec.damp)
+    assert np.max(np.abs(g["H"] - ref["H"])) <= 2e-12 * np.max(np.abs(ref["H"]))
+    nm = assert_layer_parity(g, ref)
+    return nm, g, ref
+
+
+@pytest.mark.parametrize("key", ["conv1", "layer1.0.conv2", "layer2.0.downsample", "layer4.2.conv3"])
+def test_resnet50_layers_full(key):
+    """64x147 stem (ragged columns), 64x576, 512x256 and 2048x512: whole path, every weight compared."""
+    spec = _find(wl.config3(), key)
+    nm, _, _ = _full(spec)
+    assert nm == 0
+
+
+def test_resnet50_classifier_1000_rows():
+    spec = _find(wl.config3(), "fc")            # 1000 x 2048: rows not a multiple of the row tile
+    nm, _, _ = _full(spec)
+    assert nm == 0
+
+
+@pytest.mark.parametrize("bits,key", [(8, "y255x512"), (4, "y32x108"), (8, "y64x288"), (4, "y512x2304")])
+def test_yolov5s_layers_full(bits, key):
+    """SiLU-shaped activations (negative values), N = 8192, 8- and 4-bit, 255-row heads and the 6x6 stem."""
+    spec = _find(wl.config4(bits=(bits,)), key)
+    nm, _, _ = _full(spec)
+    assert nm == 0
+
+
+@pytest.mark.parametrize("bits", [3, 8])
+def test_scaling_shape_1024_square(bits):
+    spec = _find(wl.config5(bits=(bits,), shapes=((1024, 1024),)), "1024x1024")
+    nm, _, _ = _full(spec)
+    assert nm == 0
+
+
+def _row_subset_parity(spec, sub_rows, seed):
+    """Full GPU run; oracle Hessian / inverse / scores / order in full, oracle sweep on a seeded subset of rows."""
+    W, X = wl.make_layer(spec)
+    g = gpu_layer(W, X, spec.bits, spec.damp)
+    H = oracle.hessian_accumulate(X)
+    assert np.max(np.abs(g["H"] - H)) <= 2e-12 * np.max(np.abs(H))
+    Hinv, diag, lam = oracle.prepare_hinv(H, spec.damp)
+    assert np.max(np.abs(g["Hinv"] - Hinv)) <= 1e-9 * np.max(np.abs(Hinv))
+    sc, zp = oracle.minmax_grid(W, spec.bits)
+    assert np.array_equal(g["scale"], sc) and np.array_equal(g["zero"], zp)
+    S, perm = oracle.sensitivity_order(W, diag, sc, zp, spec.bits)
+    assert np.allclose(g["S"], S, rtol=1e-9, atol=0)
+    assert np.array_equal(g["perm"], perm), "column order differs"
+    rows = np.sort(np.random.Generator(np.random.PCG64(seed)).choice(spec.rows, sub_rows, replace=False))
+    ref = oracle.quantize_layer(W[rows], Hinv, perm, sc[rows], zp[rows], spec.bits, H_undamped=H, want_prer=True)
+    nm = compare_codes(g["codes"][rows], ref)
+    num = np.linalg.norm(g["What"][rows].astype(np.float64) - ref["What"].astype(np.float64))
+    assert num <= WHAT_RTOL * np.linalg.norm(ref["What"].astype(np.float64))
+    # loss of the whole layer from its definition, 1/2 tr(dW H dW^T), with the GPU's own What (library matmul)
+    dW = W.astype(np.float64) - g["What"].astype(np.float64)
+    loss_def = 0.5 * float(np.sum((dW @ H) * dW))
+    assert abs(float(g["loss"][0]) - loss_def) <= 1e-9 * loss_def
+    # and the oracle's loss on its rows against the same definition on the GPU's rows
+    dWs = dW[rows]
+    assert abs(0.5 * float(np.sum((dWs @ H) * dWs)) - ref["loss"]) <= LOSS_RTOL * ref["loss"]
+    return nm
+
+
+def test_resnet50_512x4608_cols_exceed_calibration_columns():
+    """layer4 3x3 convolution: 4608 columns against 4096 calibration columns (rank-deficient before damping), the
+    case in which the column order is most sensitive to the accuracy of H and of its inverse."""
+    spec = _find(wl.config3(), "layer4.1.conv2")
+    assert (spec.rows, spec.cols) == (512, 4608)
+    assert _row_subset_parity(spec, 48, seed=1) == 0
+
+
+def test_yolov5s_extra_512x4608_8bit():
+    spec = _find(wl.config4(bits=(8,)), "y512x4608")
+    assert _row_subset_parity(spec, 32, seed=2) == 0
