@@ -1,0 +1,120 @@
+"""Quantizes a whole synthetic layer set, layer by layer, on one GPU and reports per-layer and per-stage device time.
+
+    python -m paper_2509_05576_b200.layer_set_run --config 3            # the 54 ResNet-50-shaped layers, 4-bit
+    python -m paper_2509_05576_b200.layer_set_run --config 4 --bits 8   # the YOLOv5s-shaped stack
+    python -m paper_2509_05576_b200.layer_set_run --config 5 --bits 4   # square / wide scaling shapes
+
+Every layer goes through the five C-ABI calls (Hessian, damped inverse, grid, scores + order, sweep); each call is
+bracketed by CUDA events on the launching stream, an L2-sized buffer is rewritten before every timed repetition.
+Stage rooflines use the algorithmic work of the stage (MAC = 2 flops): Gram cols (cols + 1) n on the int8 tensor
+pipe, inverse cols^3 (Cholesky + triangular inverse + V V^T) and sweep 4/3 cols^3 / 4 + ... on the float64 pipe --
+see ``stage_work``.  Prints a table and one JSON line with the set totals.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import ptq
+from . import workloads as wl
+
+FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
+INT8_OVER_BF16 = 2.0
+
+
+def _peaks():
+    path = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p["hbm_gbs"], p["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def stage_work(spec):
+    """Algorithmic flops per stage (MAC = 2 flops)."""
+    r, c, n = spec.rows, spec.cols, spec.n
+    return {
+        "hessian": float(c) * (c + 1) * n,                 # symmetric half of 2 X X^T
+        "inverse": float(c) ** 3,                          # Cholesky c^3/3 + triangular inverse c^3/3 + V V^T c^3/3
+        "sweep": float(c) ** 3 / 3 + float(r) * c * c + 2.0 * r * c * c,   # Cholesky of the permuted inverse, Eq. 11, loss
+    }
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--bits", type=int, default=None, help="bit-width filter for configs 4 and 5")
+    ap.add_argument("--reps", type=int, default=2)
+    ap.add_argument("--limit", type=int, default=0, help="only the first LIMIT layers (0: all)")
+    ap.add_argument("--max-cols", type=int, default=0, help="skip layers with more columns (0: none)")
+    args = ap.parse_args(argv)
+    if not torch.cuda.is_available():
+        raise RuntimeError("layer_set_run needs a CUDA device")
+    if args.config == 4:
+        specs = wl.config4(bits=(args.bits,) if args.bits else (8, 4))
+    elif args.config == 5:
+        specs = wl.config5(bits=(args.bits,) if args.bits else (3, 4, 8))
+    else:
+        specs = wl.CONFIGS[args.config]()
+    if args.max_cols:
+        specs = [s for s in specs if s.cols <= args.max_cols]
+    if args.limit:
+        specs = specs[:args.limit]
+    hbm, bf16, src = _peaks()
+    int8_peak = bf16 * INT8_OVER_BF16
+    s = torch.cuda.current_stream()
+    flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
+    ws = ptq.Workspace()
+    rows_out = []
+    totals = {"weights": 0, "ms": 0.0}
+    stage_tot = {}
+    print(f"{'layer':28s} {'rows':>5s} {'cols':>6s} {'n':>5s} {'b':>2s} {'total ms':>9s} {'Mw/s':>8s} "
+          f"{'hess':>7s} {'inv':>7s} {'order':>6s} {'sweep':>7s} {'%int8':>6s} {'%f64 inv':>8s} {'%f64 swp':>8s} {'loss':>12s}")
+    for spec in specs:
+        W, X = wl.make_layer(spec)
+        Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
+        bufs = ptq.LayerBuffers(spec.rows, spec.cols)
+        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, bufs=bufs, ws=ws, stream=s)    # warm-up
+        torch.cuda.synchronize()
+        ptq.check_status(bufs.status, spec.name)
+        per = {}
+        for rep in range(args.reps):
+            flush.fill_(rep)
+            ev = []
+            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, bufs=bufs, ws=ws, stream=s, events=ev)
+            torch.cuda.synchronize()
+            for name, a, b in ev:
+                per.setdefault(name, []).append(a.elapsed_time(b))
+        ptq.check_status(bufs.status, spec.name)
+        st = {k: float(np.median(v)) for k, v in per.items()}
+        total = sum(st.values())
+        work = stage_work(spec)
+        frac = {"hessian": work["hessian"] / (st["hessian"] * 1e-3) / 1e12 / int8_peak,
+                "inverse": work["inverse"] / (st["inverse"] * 1e-3) / 1e12 / FP64_PEAK_TFLOPS,
+                "sweep": work["sweep"] / (st["sweep"] * 1e-3) / 1e12 / FP64_PEAK_TFLOPS}
+        loss = float(bufs.loss.item())
+        print(f"{spec.name:28s} {spec.rows:5d} {spec.cols:6d} {spec.n:5d} {spec.bits:2d} {total:9.3f} "
+              f"{spec.weights / total / 1e3:8.1f} {st['hessian']:7.3f} {st['inverse']:7.3f} "
+              f"{st['grid'] + st['order']:6.3f} {st['sweep']:7.3f} {100 * frac['hessian']:6.2f} "
+              f"{100 * frac['inverse']:8.2f} {100 * frac['sweep']:8.2f} {loss:12.5g}")
+        rows_out.append({"layer": spec.name, "rows": spec.rows, "cols": spec.cols, "n": spec.n, "bits": spec.bits,
+                         "ms": total, "stages_ms": st, "roofline_frac": frac, "loss": loss})
+        totals["weights"] += spec.weights
+        totals["ms"] += total
+        for k, v in st.items():
+            stage_tot[k] = stage_tot.get(k, 0.0) + v
+        del Wd, Xd, bufs
+    print(json.dumps({"config": args.config, "layers": len(rows_out), "weights": totals["weights"],
+                      "total_ms": totals["ms"], "weights_per_s": totals["weights"] / (totals["ms"] * 1e-3),
+                      "stage_total_ms": stage_tot, "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak,
+                                                             "fp64_tflops": FP64_PEAK_TFLOPS, "source": src}}))
+    return 0
+
+
+if __name__ == "__main__":
+    raise SystemExit(main())

@@ -32,6 +32,7 @@ def main(argv=None):
     ap.add_argument("--iters", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--no-loss", action="store_true")
+    ap.add_argument("--kernels", action="store_true", help="also one pass with the library's per-kernel event profiler")
     args = ap.parse_args(argv)
 
     if not torch.cuda.is_available():
@@ -83,9 +84,17 @@ def main(argv=None):
         if it >= args.warmup:
             times.append(a.elapsed_time(b))
     ptq.check_status(st, args.stage)
+    kernels = None
+    if args.kernels:
+        ptq.profile_enable(True)
+        flush.fill_(7)
+        fn()
+        torch.cuda.synchronize()
+        kernels = {k: {"ms": round(ms, 4), "launches": cnt} for k, (ms, cnt) in ptq.profile_read().items()}
+        ptq.profile_enable(False)
     print(json.dumps({"stage": args.stage, "rows": args.rows, "cols": args.cols, "n": args.n, "bits": args.bits,
                       "xdist": args.xdist, "ms": times, "ms_median": float(np.median(times)),
-                      "loss": float(bufs.loss.item()) if want_loss else None}))
+                      "loss": float(bufs.loss.item()) if want_loss else None, "kernels": kernels}))
     return 0
 
 
