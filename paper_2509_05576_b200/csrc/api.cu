@@ -192,12 +192,11 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     unsigned* bar = cv.take<unsigned>(2);
     { Launch l(K_LAMBDA, stream); lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status); }
     { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out); }
-    int st = cholesky_upper(R, n, bar, status, stream);
-    if (st) return st;
+    // W = U^-T comes out of the factorisation sweep itself (V must start as zero)
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
-    st = trtri_upper(R, V, Hinv, n, stream);
+    int st = cholesky_upper(R, n, V, bar, status, stream);
     if (st) return st;
-    st = lauum_upper(V, Hinv, n, stream);
+    st = lauum_lower(V, Hinv, n, stream);
     if (st) return st;
     { Launch l(K_EXTRACT_DIAG, stream); extract_diag_kernel<<<cdiv(n, 256), 256, 0, stream>>>(Hinv, n, Hinv_diag); }
     return launch_status();
@@ -289,7 +288,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     { Launch l(K_PERM_CHECK, stream); perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status); }
     { Launch l(K_GATHER_SYM, stream); gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U); }
     { Launch l(K_GATHER_W, stream); gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp); }
-    int st = cholesky_upper(U, n, bar, status, stream);   // blocked Eq. 12
+    int st = cholesky_upper(U, n, nullptr, bar, status, stream);   // blocked Eq. 12
     if (st) return st;
 
     st = sweep_launch(Wp, U, E, codes_p, scale, zero, rows, n, bits, sweep_flags, status, stream);

@@ -1,5 +1,5 @@
 // Float64 blocked factorisation pieces: A = U^T U (upper Cholesky, in place, row-major), the inverse of the
-// factor by recursive halving, and Hinv = V V^T.  Sec. 5 item 1 of the paper (Cholesky, then the inverse of
+// factor W = U^-T from the same sweep, and Hinv = W^T W.  Sec. 5 item 1 of the paper (Cholesky, then the inverse of
 // the factor); the same Cholesky applied to the permuted inverse Hessian is the blocked form of Eq. 12:
 // step p of a right-looking Cholesky subtracts (row p)^T (row p) / pivot from the trailing matrix.
 #pragma once
@@ -93,22 +93,23 @@ __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gsrc, 
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(gsrc), "r"(sz) : "memory");
 }
 
-// Loads the 64 x ncols block A[r0 .. r0+63][c0 .. c0+ncols-1] into dst[64][kCholLd]; entries beyond n are zero.
+// Loads the 64 x ncols block A[r0 .. r0+63][c0 .. c0+ncols-1] into dst[64][kCholLd], ncols = 1 << lg in {16, 32, 64};
+// entries beyond n are zero.
 __device__ __forceinline__ void chol_load_block(double* dst, const double* __restrict__ A, int64_t ld, int n, int r0,
-                                                int c0, int ncols, int vec16) {
+                                                int c0, int lg, int vec16) {
+    const double* base = A + (int64_t)r0 * ld + c0;
     if (vec16) {
-        for (int idx = threadIdx.x; idx < kNB * kNB / 2; idx += kCholThreads) {
-            const int r = idx >> 5, c = (idx & 31) * 2;
-            if (c >= ncols) continue;
+        const int sh = lg - 1;                           // pairs per row = 1 << sh
+        for (int idx = threadIdx.x; idx < (kNB << sh); idx += kCholThreads) {
+            const int r = idx >> sh, c = (idx & ((1 << sh) - 1)) * 2;
             const bool ok = r0 + r < n && c0 + c < n;      // n is even on this path: a pair never straddles n
-            cp_async16_cg(dst + r * kCholLd + c, ok ? A + (int64_t)(r0 + r) * ld + c0 + c : A, ok);
+            cp_async16_cg(dst + r * kCholLd + c, ok ? base + (int64_t)r * ld + c : A, ok);
         }
     } else {
-        for (int idx = threadIdx.x; idx < kNB * kNB; idx += kCholThreads) {
-            const int r = idx >> 6, c = idx & 63;
-            if (c >= ncols) continue;
+        for (int idx = threadIdx.x; idx < (kNB << lg); idx += kCholThreads) {
+            const int r = idx >> lg, c = idx & ((1 << lg) - 1);
             const bool ok = r0 + r < n && c0 + c < n;
-            cp_async8(dst + r * kCholLd + c, ok ? A + (int64_t)(r0 + r) * ld + c0 + c : A, ok);
+            cp_async8(dst + r * kCholLd + c, ok ? base + (int64_t)r * ld + c : A, ok);
         }
     }
 }
@@ -218,18 +219,21 @@ __device__ __forceinline__ void chol_strip_blocks(double (&acc)[8][2][2], double
     (chol_strip_block<Bs>(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, reporter, status), ...);
 }
 
-// Factorises the diagonal block at k0 and, when chunk >= 0, the 64 panel columns starting at
-// k0 + 64 + 64 * chunk with it.  The diagonal factor is written only when write_diag is set.
-__device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, int n, int k0, int chunk,
-                                           bool write_diag, double* smem, int vec16, int32_t* status) {
+// Factorises the diagonal block of A at k0 and applies the same row operations to 64 panel columns with it: columns
+// pc0 .. pc0 + 63 of rows k0 .. k0 + 63 of the matrix P (row stride ld), or, when `identity` is set, of the identity
+// block (whose transform is the inverse of the transposed diagonal factor).  P == nullptr: diagonal block only.  The
+// diagonal factor is written only when write_diag is set.
+__device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, int n, int k0, double* __restrict__ P,
+                                           int pc0, bool identity, bool write_diag, double* smem, int vec16,
+                                           int32_t* status) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int lq = lane >> 2, lr = lane & 3;
     double* Rbuf = smem;
     double* Ubuf = smem + 8 * kStripLd;
     double* Wbuf = smem + 2 * 8 * kStripLd;
     const bool is_diag = warp < 4;
-    const int gc0 = is_diag ? k0 + 16 * warp : k0 + kNB + chunk * kNB + 16 * (warp - 4);   // first global column
-    const int sc0 = 16 * warp;                                                               // first strip column
+    const int gc0 = is_diag ? k0 + 16 * warp : pc0 + 16 * (warp - 4);       // first global column of this warp
+    const int sc0 = 16 * warp;                                               // first strip column
     double acc[8][2][2];
 #pragma unroll
     for (int rb = 0; rb < 8; ++rb)
@@ -245,15 +249,16 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
                         if (grow < n && gc < n) val = __ldcg(A + (int64_t)grow * ld + gc);
                         else if (sc == row) val = 1.0;                   // identity padding below n
                     }
-                } else if (chunk >= 0 && grow < n && gc < n) {
-                    val = __ldcg(A + (int64_t)grow * ld + gc);
+                } else if (P != nullptr && grow < n && gc < n) {
+                    val = identity ? (sc - kNB == row ? 1.0 : 0.0) : __ldcg(P + (int64_t)grow * ld + gc);
                 }
                 acc[rb][cb][e] = val;
             }
         }
     chol_strip_blocks(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, write_diag && threadIdx.x == 0, status,
                       std::make_integer_sequence<int, 8>());
-    if (is_diag ? write_diag : chunk >= 0) {
+    if (is_diag ? write_diag : P != nullptr) {
+        double* M = is_diag ? A : P;
 #pragma unroll
         for (int rb = 0; rb < 8; ++rb)
 #pragma unroll
@@ -261,7 +266,7 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
                 const int row = 8 * rb + lq, grow = k0 + row;
                 const int sc = sc0 + 8 * cb + 2 * lr, gc = gc0 + 8 * cb + 2 * lr;
                 if (grow >= n || gc >= n) continue;
-                double* dst = A + (int64_t)grow * ld + gc;
+                double* dst = M + (int64_t)grow * ld + gc;
                 const bool keep0 = !is_diag || sc >= row, keep1 = !is_diag || sc + 1 >= row;
                 if (vec16 && keep0) {
                     __stcg(reinterpret_cast<double2*>(dst), make_double2(acc[rb][cb][0], acc[rb][cb][1]));
@@ -273,69 +278,74 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
     }
 }
 
-// One H x 64 piece of a trailing tile: rows [h0, h0 + H) of tile (bi, bj), operands in shared memory.
+// One H x 64 piece of a trailing tile: C[i0 .. i0 + H)[j0 .. j0 + 64) -= as^T bs with the operands in shared memory
+// (as[kk][r], bs[kk][c]); eight warps as 2 x 4, each (H / 2) x 16.  tri_off >= 0: the piece lies in a diagonal tile
+// and only entries with c >= tri_off + r are touched.
 template <int H>
-__device__ __forceinline__ void chol_trailing_piece(double* __restrict__ A, int64_t ld, int n, const double* as,
-                                                    const double* bs, int bi, int bj, int h0, int vec16) {
-    constexpr int FM = H / 16;
+__device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int64_t ld, int n, const double* as,
+                                                    const double* bs, int i0, int j0, int tri_off, int vec16) {
+    constexpr int FM = H / 16, FN = 2;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int wm0 = (warp >> 2) * (H / 2), wn0 = (warp & 3) * 16;
     const int lq = lane >> 2, lr = lane & 3;
-    const int i0 = bi * kNB + h0, j0 = bj * kNB;
-    // the old values of the tile are fetched first, so that their latency hides behind the MMAs
-    double acc[FM][2][2];
-    bool keep[FM][2][2];
+    // the old values of the tile are requested first and only consumed after the MMA loop, so that their latency
+    // hides behind it
+    double old[FM][FN][2], acc[FM][FN][2];
+    bool keep[FM][FN][2];
 #pragma unroll
     for (int a = 0; a < FM; ++a) {
         const int r = wm0 + a * 8 + lq;
 #pragma unroll
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < FN; ++b) {
             const int c = wn0 + b * 8 + 2 * lr;
             const bool in = i0 + r < n && j0 + c < n;
-            keep[a][b][0] = in && (bi != bj || c >= h0 + r);
-            keep[a][b][1] = in && j0 + c + 1 < n && (bi != bj || c + 1 >= h0 + r);
-            const double* src = A + (int64_t)(i0 + r) * ld + j0 + c;
+            keep[a][b][0] = in && (tri_off < 0 || c >= tri_off + r);
+            keep[a][b][1] = in && j0 + c + 1 < n && (tri_off < 0 || c + 1 >= tri_off + r);
+            const double* src = C + (int64_t)(i0 + r) * ld + j0 + c;
             if (vec16 && keep[a][b][0]) {             // n even: the pair is inside; keep[0] implies keep[1]
                 const double2 v = __ldcg(reinterpret_cast<const double2*>(src));
-                acc[a][b][0] = v.x;
-                acc[a][b][1] = v.y;
+                old[a][b][0] = v.x;
+                old[a][b][1] = v.y;
             } else {
-                acc[a][b][0] = keep[a][b][0] ? __ldcg(src) : 0.0;
-                acc[a][b][1] = keep[a][b][1] ? __ldcg(src + 1) : 0.0;
+                old[a][b][0] = keep[a][b][0] ? __ldcg(src) : 0.0;
+                old[a][b][1] = keep[a][b][1] ? __ldcg(src + 1) : 0.0;
             }
+            acc[a][b][0] = acc[a][b][1] = 0.0;
         }
     }
 #pragma unroll 4
     for (int kk = 0; kk < kNB; kk += 4) {
-        double af[FM], bf[2];
+        double af[FM], bf[FN];
 #pragma unroll
-        for (int a = 0; a < FM; ++a) af[a] = -as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
+        for (int a = 0; a < FM; ++a) af[a] = as[(kk + lr) * kCholLd + wm0 + a * 8 + lq];
 #pragma unroll
-        for (int b = 0; b < 2; ++b) bf[b] = bs[(kk + lr) * kCholLd + wn0 + b * 8 + lq];
+        for (int b = 0; b < FN; ++b) bf[b] = bs[(kk + lr) * kCholLd + wn0 + b * 8 + lq];
 #pragma unroll
         for (int a = 0; a < FM; ++a)
 #pragma unroll
-            for (int b = 0; b < 2; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+            for (int b = 0; b < FN; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
     }
 #pragma unroll
     for (int a = 0; a < FM; ++a) {
         const int r = wm0 + a * 8 + lq;
 #pragma unroll
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < FN; ++b) {
             const int c = wn0 + b * 8 + 2 * lr;
-            double* dst = A + (int64_t)(i0 + r) * ld + j0 + c;
+            double* dst = C + (int64_t)(i0 + r) * ld + j0 + c;
+            const double v0 = old[a][b][0] - acc[a][b][0], v1 = old[a][b][1] - acc[a][b][1];
             if (vec16 && keep[a][b][0]) {
-                __stcg(reinterpret_cast<double2*>(dst), make_double2(acc[a][b][0], acc[a][b][1]));
+                __stcg(reinterpret_cast<double2*>(dst), make_double2(v0, v1));
             } else {
-                if (keep[a][b][0]) __stcg(dst, acc[a][b][0]);
-                if (keep[a][b][1]) __stcg(dst + 1, acc[a][b][1]);
+                if (keep[a][b][0]) __stcg(dst, v0);
+                if (keep[a][b][1]) __stcg(dst + 1, v1);
             }
         }
     }
 }
 
 __global__ void __launch_bounds__(kCholThreads, 1)
-chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned* bar, int32_t* status) {
+chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t ld, int vec16, unsigned* bar,
+                 int32_t* status) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
     int* s_flag = reinterpret_cast<int*>(opnd + 2 * 2 * kNB * kCholLd);     // the strip panels alias opnd
@@ -347,11 +357,19 @@ chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned*
     for (int k = 0; k < nb; ++k) {
         const int k0 = k * kNB;
         // ------------------------------------------------------------------ strip phase
-        const int panel_cols = n - k0 - kNB;                                // columns to the right of the block
-        const int chunks = panel_cols > 0 ? (panel_cols + kNB - 1) / kNB : 0;
-        const int reps = chunks > 0 ? chunks : 1;                            // last block: diagonal only
+        // work items: the panel chunks of A right of the block, then (with Wm) the chunks 0 .. k of row block k of W,
+        // the last of which starts as the identity
+        const int chunksA = nb - 1 - k;
+        const int chunksW = Wm != nullptr ? k + 1 : 0;
+        const int items = chunksA + chunksW;
+        const int reps = items > 0 ? items : 1;                              // last block without Wm: diagonal only
         for (int g = blockIdx.x; g < reps; g += G) {
-            chol_strip(A, ld, n, k0, chunks > 0 ? g : -1, g == 0, opnd, vec16, status);
+            double* P = nullptr;
+            int pc0 = 0;
+            bool ident = false;
+            if (g < chunksA) { P = A; pc0 = k0 + kNB + g * kNB; }
+            else if (g < items) { P = Wm; pc0 = (g - chunksA) * kNB; ident = (g - chunksA) == k; }
+            chol_strip(A, ld, n, k0, P, pc0, ident, g == 0, opnd, vec16, status);
             __syncthreads();     // the panel buffers are reused by the next repetition and by the trailing phase
         }
         if (k == nb - 1) break;
@@ -359,43 +377,67 @@ chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned*
         if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
 
         // ------------------------------------------------------------------ trailing phase
+        // tiles of A: (i, j), k < i <= j: A[i][j] -= U[k][i]^T U[k][j]; tiles of W: (i, c), k < i, c <= k:
+        // W[i][c] -= U[k][i]^T W[k][c].  Row-major lists, A first.
         const int m = nb - 1 - k;
-        const int T = m * (m + 1) / 2;
+        const int TA = m * (m + 1) / 2;
+        const int TW = Wm != nullptr ? m * (k + 1) : 0;
+        const int T = TA + TW;
         // tiles are cut into 64 / H row pieces so that a short tile list still spreads over the grid
-        const int H = 4 * T <= G ? 16 : (2 * T <= G ? 32 : 64);
-        const int pieces = kNB / H;
-        const int TP = T * pieces;
-        auto piece_coords = [&](int tp, int& bi, int& bj, int& h0) {
-            const int t = tp / pieces;
-            h0 = (tp - t * pieces) * H;
-            int i = k + 1, rem = t;
-            while (rem >= nb - i) { rem -= nb - i; ++i; }
-            bi = i; bj = i + rem;
+        const int lgH = 4 * T <= G ? 4 : (2 * T <= G ? 5 : 6);
+        const int lgP = 6 - lgH;
+        const int TP = T << lgP;
+        struct Piece { double* C; const double* Bsrc; int i0, j0, bcol, tri; };
+        auto piece_of = [&](int tp) {
+            Piece pc;
+            const int t = tp >> lgP;
+            const int h0 = (tp & ((1 << lgP) - 1)) << lgH;
+            if (t < TA) {
+                // largest r with r m - r (r - 1) / 2 <= t
+                const float mm = (float)m + 0.5f;
+                int r = (int)(mm - sqrtf(fmaxf(mm * mm - 2.0f * (float)t, 0.0f)));
+                r = r < 0 ? 0 : (r > m - 1 ? m - 1 : r);
+                while (r > 0 && r * m - r * (r - 1) / 2 > t) --r;
+                while (r + 1 < m && (r + 1) * m - (r + 1) * r / 2 <= t) ++r;
+                const int bi = k + 1 + r, bj = bi + (t - (r * m - r * (r - 1) / 2));
+                pc.C = A; pc.Bsrc = A; pc.i0 = bi * kNB + h0; pc.j0 = bj * kNB; pc.bcol = bj * kNB;
+                pc.tri = bi == bj ? h0 : -1;
+            } else {
+                const int tw = t - TA;
+                const int r = tw / (k + 1), c = tw - r * (k + 1);
+                pc.C = Wm; pc.Bsrc = Wm; pc.i0 = (k + 1 + r) * kNB + h0; pc.j0 = c * kNB; pc.bcol = c * kNB;
+                pc.tri = -1;
+            }
+            return pc;
         };
-        auto load_piece = [&](int tp, int stg) {
-            int bi, bj, h0;
-            piece_coords(tp, bi, bj, h0);
+        auto load_piece = [&](const Piece& pc, int stg) {
             double* dst = opnd + stg * 2 * kNB * kCholLd;
-            chol_load_block(dst, A, ld, n, k0, bi * kNB + h0, H, vec16);
-            chol_load_block(dst + kNB * kCholLd, A, ld, n, k0, bj * kNB, kNB, vec16);
+            chol_load_block(dst, A, ld, n, k0, pc.i0, lgH, vec16);                     // U[k0 + kk][i0 + r]
+            chol_load_block(dst + kNB * kCholLd, pc.Bsrc, ld, n, k0, pc.bcol, 6, vec16);   // U or W [k0 + kk][j0 + c]
         };
         int stage = 0;
-        if ((int)blockIdx.x < TP) load_piece(blockIdx.x, 0);
+        Piece cur{}, nxt{};
+        if ((int)blockIdx.x < TP) {
+            cur = piece_of(blockIdx.x);
+            load_piece(cur, 0);
+        }
         cp_async_commit();
         for (int tp = blockIdx.x; tp < TP; tp += G) {
-            if (tp + G < TP) load_piece(tp + G, stage ^ 1);
+            if (tp + G < TP) {
+                nxt = piece_of(tp + G);
+                load_piece(nxt, stage ^ 1);
+            }
             cp_async_commit();
             cp_async_wait<1>();
             __syncthreads();
-            int bi, bj, h0;
-            piece_coords(tp, bi, bj, h0);
-            const double* as = opnd + stage * 2 * kNB * kCholLd;            // as[kk][m] = U[k0 + kk][i0 + h0 + m]
-            const double* bs = as + kNB * kCholLd;                           // bs[kk][c] = U[k0 + kk][j0 + c]
-            if (H == 64) chol_trailing_piece<64>(A, ld, n, as, bs, bi, bj, h0, vec16);
-            else if (H == 32) chol_trailing_piece<32>(A, ld, n, as, bs, bi, bj, h0, vec16);
-            else chol_trailing_piece<16>(A, ld, n, as, bs, bi, bj, h0, vec16);
+            const double* as = opnd + stage * 2 * kNB * kCholLd;
+            const double* bs = as + kNB * kCholLd;
+            if (lgH == 6) chol_trailing_piece<64>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
+            else if (lgH == 5) chol_trailing_piece<32>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
+            else chol_trailing_piece<16>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
             __syncthreads();     // all warps are done with this stage before it is refilled
             stage ^= 1;
+            cur = nxt;
         }
         cp_async_wait<0>();
         ++epoch;
@@ -405,9 +447,11 @@ chol_coop_kernel(double* __restrict__ A, int n, int64_t ld, int vec16, unsigned*
     if (tid == 0 && ld_acquire_u32(&bar[1]) != 0u) report(status, PTQ_ERR_TIMEOUT, blockIdx.x, 1);
 }
 
-// In-place blocked upper Cholesky of the n x n matrix A (row stride n).  Only the upper triangle is read or
-// written.  `bar` is 2 x uint32 of device scratch.
-inline int cholesky_upper(double* A, int n, unsigned* bar, int32_t* status, cudaStream_t stream) {
+// In-place blocked upper Cholesky A = U^T U of the n x n matrix A (row stride n).  Only the upper triangle is read or
+// written.  With Wm (n x n, zero on entry) the same sweep also leaves W = U^-T there (lower triangular): the row
+// operations of the factorisation are applied to the identity, Sec. 5 item 1's "inverse of the decomposed result".
+// `bar` is 2 x uint32 of device scratch.
+inline int cholesky_upper(double* A, int n, double* Wm, unsigned* bar, int32_t* status, cudaStream_t stream) {
     static int grid = 0;
     if (grid == 0) {
         if (cudaFuncSetAttribute(chol_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -425,8 +469,8 @@ inline int cholesky_upper(double* A, int n, unsigned* bar, int32_t* status, cuda
     }
     if (cudaMemsetAsync(bar, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int64_t ld = n;
-    int vec16 = ((n & 1) == 0 && aligned16(A)) ? 1 : 0;
-    void* args[] = {&A, &n, &ld, &vec16, &bar, &status};
+    int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;
+    void* args[] = {&A, &Wm, &n, &ld, &vec16, &bar, &status};
     Launch l(K_CHOL_COOP, stream);
     if (cudaLaunchCooperativeKernel((const void*)chol_coop_kernel, dim3(grid), dim3(kCholThreads), args,
                                     kCholSmemBytes, stream) != cudaSuccess) {
@@ -436,70 +480,12 @@ inline int cholesky_upper(double* A, int n, unsigned* bar, int32_t* status, cuda
     return PTQ_OK;
 }
 
-// V[b, b] = inverse of the upper-triangular diagonal block R[b, b]; one CTA per 64-block, one thread per column.
-__global__ void __launch_bounds__(kNB) diag_inverse_kernel(const double* __restrict__ R, double* __restrict__ V,
-                                                            int64_t ld, int n) {
-    __shared__ double Us[kNB][kNB];
-    const int b0 = blockIdx.x * kNB;
-    const int kb = n - b0 < kNB ? n - b0 : kNB;
-    for (int idx = threadIdx.x; idx < kNB * kNB; idx += kNB) {
-        const int r = idx >> 6, c = idx & 63;
-        double v = (r == c) ? 1.0 : 0.0;
-        if (r < kb && c < kb && c >= r) v = R[(int64_t)(b0 + r) * ld + b0 + c];
-        Us[r][c] = v;
-    }
-    __syncthreads();
-    const int j = threadIdx.x;
-    double v[kNB];
-#pragma unroll
-    for (int i = kNB - 1; i >= 0; --i) {
-        double s = (i == j) ? 1.0 : 0.0;
-#pragma unroll
-        for (int k = i + 1; k < kNB; ++k) s = fma(-Us[i][k], v[k], s);
-        v[i] = s / Us[i][i];
-    }
-    if (j < kb) {
-#pragma unroll
-        for (int i = 0; i < kNB; ++i)
-            if (i <= j) V[(int64_t)(b0 + i) * ld + b0 + j] = v[i];
-    }
-}
-
-// V = R^-1 for upper-triangular R (n x n).  V must be zero on entry; T is n x n scratch.
-// Recursive halving: with R = [R11 R12; 0 R22], V12 = -V11 (R12 V22); all pairs of one level run as one batch.
-inline int trtri_upper(const double* R, double* V, double* T, int n, cudaStream_t stream) {
-    { Launch l(K_DIAG_INVERSE, stream); diag_inverse_kernel<<<cdiv(n, kNB), kNB, 0, stream>>>(R, V, n, n); }
-    for (int64_t s = kNB; s < n; s *= 2) {
-        const int pairs = (int)((n + 2 * s - 1) / (2 * s));
-        const int64_t step = 2 * s * ((int64_t)n + 1);
-        GemmParams g = gemm_defaults();     // T12 = R12 V22   (V22 upper: k stops at the tile's last column)
-        g.A = R + s; g.lda = n; g.a_trans = 0; g.batch_a = step;
-        g.B = V + s * ((int64_t)n + 1); g.ldb = n; g.b_trans = 0; g.batch_b = step;
-        g.C = T + s; g.ldc = n; g.batch_c = step;
-        g.M = (int)s; g.N = (int)s; g.K = (int)s;
-        g.ragN_lim = n - (int)s; g.ragN_step = (int)(2 * s); g.k_is_n = 1;
-        g.kend_mode = 1;
-        int st = launch_dgemm(K_DGEMM_TRTRI, g, pairs, stream);
-        if (st) return st;
-        GemmParams h = gemm_defaults();     // V12 = -V11 T12   (V11 upper: k starts at the tile's first row)
-        h.A = V; h.lda = n; h.a_trans = 0; h.batch_a = step;
-        h.B = T + s; h.ldb = n; h.b_trans = 0; h.batch_b = step;
-        h.C = V + s; h.ldc = n; h.batch_c = step;
-        h.M = (int)s; h.N = (int)s; h.K = (int)s;
-        h.ragN_lim = n - (int)s; h.ragN_step = (int)(2 * s);
-        h.kbeg_mode = 2;
-        h.alpha = -1.0;
-        st = launch_dgemm(K_DGEMM_TRTRI, h, pairs, stream);
-        if (st) return st;
-    }
-    return launch_status();
-}
-
-// Hinv = V V^T for upper-triangular V: the sum over k starts at max(i, j); upper tiles computed, mirrored below.
-inline int lauum_upper(const double* V, double* Hinv, int n, cudaStream_t stream) {
+// Hinv = W^T W for the lower-triangular W = U^-T: Hinv[i][j] = sum over k >= max(i, j) of W[k][i] W[k][j]; upper tiles
+// computed, mirrored below.
+inline int lauum_lower(const double* W, double* Hinv, int n, cudaStream_t stream) {
     GemmParams g = gemm_defaults();
-    g.A = V; g.lda = n; g.a_trans = 0;
-    g.B = V; g.ldb = n; g.b_trans = 1;
+    g.A = W; g.lda = n; g.a_trans = 1;
+    g.B = W; g.ldb = n; g.b_trans = 0;
     g.C = Hinv; g.ldc = n;
     g.M = n; g.N = n; g.K = n;
     g.kbeg_mode = 1; g.upper_only = 1; g.mirror = 1;

@@ -331,14 +331,22 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                     }
                 cp_async_wait<0>();
                 __syncthreads();
+                double prod[4][2];
+#pragma unroll
+                for (int a = 0; a < 4; ++a) prod[a][0] = prod[a][1] = 0.0;
 #pragma unroll 4
                 for (int kk = 0; kk < kNB; kk += 4) {
                     const double bf = Bb[(kk + lr) * kSweepLd + 8 * warp + lq];
 #pragma unroll
                     for (int a = 0; a < 4; ++a) {
-                        const double af = -Ea[(8 * a + lq) * kSweepLd + kk + lr];
-                        dmma_884(blk[a][0], blk[a][1], af, bf);
+                        const double af = Ea[(8 * a + lq) * kSweepLd + kk + lr];
+                        dmma_884(prod[a][0], prod[a][1], af, bf);
                     }
+                }
+#pragma unroll
+                for (int a = 0; a < 4; ++a) {
+                    blk[a][0] -= prod[a][0];
+                    blk[a][1] -= prod[a][1];
                 }
                 prepared = true;
                 continue;
@@ -361,7 +369,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                     cp_async_commit();
                     // old values of the tile first (their latency hides behind the MMAs)
                     const int j0 = bp * kNB;
-                    double acc[2][2][2];
+                    double old[2][2][2], acc[2][2][2];
                     bool keep[2][2][2];
 #pragma unroll
                     for (int a = 0; a < 2; ++a) {
@@ -374,12 +382,13 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                             const double* src = prm.Wp + (int64_t)r * n + c;
                             if (prm.vec16 && keep[a][q][0]) {
                                 const double2 v = __ldcg(reinterpret_cast<const double2*>(src));
-                                acc[a][q][0] = v.x;
-                                acc[a][q][1] = v.y;
+                                old[a][q][0] = v.x;
+                                old[a][q][1] = v.y;
                             } else {
-                                acc[a][q][0] = keep[a][q][0] ? __ldcg(src) : 0.0;
-                                acc[a][q][1] = keep[a][q][1] ? __ldcg(src + 1) : 0.0;
+                                old[a][q][0] = keep[a][q][0] ? __ldcg(src) : 0.0;
+                                old[a][q][1] = keep[a][q][1] ? __ldcg(src + 1) : 0.0;
                             }
+                            acc[a][q][0] = acc[a][q][1] = 0.0;
                         }
                     }
                     cp_async_wait<1>();
@@ -389,7 +398,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                     for (int kk = 0; kk < kNB; kk += 4) {
                         double af[2], bf[2];
 #pragma unroll
-                        for (int a = 0; a < 2; ++a) af[a] = -Ea[(wm0 + a * 8 + lq) * kSweepLd + kk + lr];
+                        for (int a = 0; a < 2; ++a) af[a] = Ea[(wm0 + a * 8 + lq) * kSweepLd + kk + lr];
 #pragma unroll
                         for (int q = 0; q < 2; ++q) bf[q] = bs[(kk + lr) * kSweepLd + wn0 + q * 8 + lq];
 #pragma unroll
@@ -404,11 +413,12 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         for (int q = 0; q < 2; ++q) {
                             const int c = j0 + wn0 + q * 8 + 2 * lr;
                             double* dst = prm.Wp + (int64_t)r * n + c;
+                            const double v0 = old[a][q][0] - acc[a][q][0], v1 = old[a][q][1] - acc[a][q][1];
                             if (prm.vec16 && keep[a][q][0]) {
-                                __stcg(reinterpret_cast<double2*>(dst), make_double2(acc[a][q][0], acc[a][q][1]));
+                                __stcg(reinterpret_cast<double2*>(dst), make_double2(v0, v1));
                             } else {
-                                if (keep[a][q][0]) __stcg(dst, acc[a][q][0]);
-                                if (keep[a][q][1]) __stcg(dst + 1, acc[a][q][1]);
+                                if (keep[a][q][0]) __stcg(dst, v0);
+                                if (keep[a][q][1]) __stcg(dst + 1, v1);
                             }
                         }
                     }
