@@ -51,6 +51,8 @@ __global__ void damp_copy_kernel(const double* __restrict__ H, double* __restric
 //                  (see chol_strip).  That replaces "factor the block, then solve the panel against it".
 //   trailing phase A[i][j] -= U[k][i]^T U[k][j] on the upper 64 x 64 tiles, float64 tensor-core MMA, operands
 //                  double-buffered through shared memory with cp.async.
+// When the next block row has few strip work items, a few CTAs update and factorise it (look-ahead) while the others
+// are still applying the current one to the rows below, which takes the strip off the critical path.
 // The phases are separated by a grid-wide barrier whose wait is bounded: when it expires the CTA records
 // PTQ_ERR_TIMEOUT, raises the abort word and leaves; the other CTAs see the abort word and leave too.
 // A non-positive or non-finite pivot is reported (PTQ_ERR_NOT_SPD, pivot index) and replaced by 1.
@@ -206,6 +208,7 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
             const double n1 = -Ubuf[(4 + lr) * kStripLd + 8 * r + lq];
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
+                if (warp < 4 && 8 * r > c0 + 8 * cb + 7) continue;       // entirely below the diagonal: never used
                 dmma_884(acc[r][cb][0], acc[r][cb][1], n0, bf[cb][0]);
                 dmma_884(acc[r][cb][0], acc[r][cb][1], n1, bf[cb][1]);
             }
@@ -223,9 +226,12 @@ __device__ __forceinline__ void chol_strip_blocks(double (&acc)[8][2][2], double
 // pc0 .. pc0 + 63 of rows k0 .. k0 + 63 of the matrix P (row stride ld), or, when `identity` is set, of the identity
 // block (whose transform is the inverse of the transposed diagonal factor).  P == nullptr: diagonal block only.  The
 // diagonal factor is written only when write_diag is set.
+// When upd_a is given, the strip is first brought up to date with the previous block row (look-ahead):
+//     strip -= upd_a^T [upd_a | upd_b],   upd_a[kk][r] = U[k0 - 64 + kk][k0 + r],  upd_b[kk][c] = P[k0 - 64 + kk][pc0 + c]
+// (both 64 x 64 in shared memory, row stride kCholLd; upd_b == nullptr: the panel part needs no update).
 __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, int n, int k0, double* __restrict__ P,
                                            int pc0, bool identity, bool write_diag, double* smem, int vec16,
-                                           int32_t* status) {
+                                           int32_t* status, const double* upd_a, const double* upd_b) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int lq = lane >> 2, lr = lane & 3;
     double* Rbuf = smem;
@@ -255,6 +261,41 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
                 acc[rb][cb][e] = val;
             }
         }
+    if (upd_a != nullptr) {
+        cp_async_wait<0>();
+        __syncthreads();
+        const double* bsrc = is_diag ? upd_a + 16 * warp : (upd_b != nullptr ? upd_b + 16 * (warp - 4) : nullptr);
+        if (bsrc != nullptr) {
+            double prod[8][2][2];
+#pragma unroll
+            for (int rb = 0; rb < 8; ++rb)
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) prod[rb][cb][0] = prod[rb][cb][1] = 0.0;
+#pragma unroll 2
+            for (int kk = 0; kk < kNB; kk += 4) {
+                double bf[2];
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) bf[cb] = bsrc[(kk + lr) * kCholLd + 8 * cb + lq];
+#pragma unroll
+                for (int rb = 0; rb < 8; ++rb) {
+                    const double af = upd_a[(kk + lr) * kCholLd + 8 * rb + lq];
+#pragma unroll
+                    for (int cb = 0; cb < 2; ++cb) {
+                        // fragments of the diagonal block that lie entirely below the diagonal are never used
+                        if (is_diag && 8 * rb > sc0 + 8 * cb + 7) continue;
+                        dmma_884(prod[rb][cb][0], prod[rb][cb][1], af, bf[cb]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int rb = 0; rb < 8; ++rb)
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    acc[rb][cb][0] -= prod[rb][cb][0];
+                    acc[rb][cb][1] -= prod[rb][cb][1];
+                }
+        }
+    }
     chol_strip_blocks(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, write_diag && threadIdx.x == 0, status,
                       std::make_integer_sequence<int, 8>());
     if (is_diag ? write_diag : P != nullptr) {
@@ -354,40 +395,42 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t
     const int nb = (n + kNB - 1) / kNB;
     unsigned epoch = 0;
 
-    for (int k = 0; k < nb; ++k) {
-        const int k0 = k * kNB;
-        // ------------------------------------------------------------------ strip phase
-        // work items: the panel chunks of A right of the block, then (with Wm) the chunks 0 .. k of row block k of W,
-        // the last of which starts as the identity
+    // strip work items of block row k: the panel chunks of A right of the block, then (with Wm) the chunks 0 .. k of
+    // row block k of W, the last of which starts as the identity
+    auto strip_items = [&](int k) { return (nb - 1 - k) + (Wm != nullptr ? k + 1 : 0); };
+    auto strip_item = [&](int k, int g, double*& P, int& pc0, bool& ident) {
         const int chunksA = nb - 1 - k;
-        const int chunksW = Wm != nullptr ? k + 1 : 0;
-        const int items = chunksA + chunksW;
+        P = nullptr; pc0 = 0; ident = false;
+        if (g < chunksA) { P = A; pc0 = (k + 1 + g) * kNB; }
+        else if (g < strip_items(k)) { P = Wm; pc0 = (g - chunksA) * kNB; ident = (g - chunksA) == k; }
+    };
+    // plain strip phase of block row k over the whole grid
+    auto strip_phase = [&](int k) {
+        const int items = strip_items(k);
         const int reps = items > 0 ? items : 1;                              // last block without Wm: diagonal only
         for (int g = blockIdx.x; g < reps; g += G) {
-            double* P = nullptr;
-            int pc0 = 0;
-            bool ident = false;
-            if (g < chunksA) { P = A; pc0 = k0 + kNB + g * kNB; }
-            else if (g < items) { P = Wm; pc0 = (g - chunksA) * kNB; ident = (g - chunksA) == k; }
-            chol_strip(A, ld, n, k0, P, pc0, ident, g == 0, opnd, vec16, status);
+            double* P; int pc0; bool ident;
+            strip_item(k, g, P, pc0, ident);
+            chol_strip(A, ld, n, k * kNB, P, pc0, ident, g == 0, opnd, vec16, status, nullptr, nullptr);
             __syncthreads();     // the panel buffers are reused by the next repetition and by the trailing phase
         }
-        if (k == nb - 1) break;
-        ++epoch;
-        if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
-
-        // ------------------------------------------------------------------ trailing phase
-        // tiles of A: (i, j), k < i <= j: A[i][j] -= U[k][i]^T U[k][j]; tiles of W: (i, c), k < i, c <= k:
-        // W[i][c] -= U[k][i]^T W[k][c].  Row-major lists, A first.
-        const int m = nb - 1 - k;
+    };
+    // Trailing tiles of block row k restricted to target rows >= row_base, processed by the CTAs cta_first .. G - 1.
+    //   tiles of A: (i, j), row_base <= i <= j: A[i][j] -= U[k][i]^T U[k][j]
+    //   tiles of W: (i, c), row_base <= i, c <= k:  W[i][c] -= U[k][i]^T W[k][c]       (row-major lists, A first)
+    auto trailing_phase = [&](int k, int row_base, int cta_first) {
+        const int k0 = k * kNB;
+        const int m = nb - row_base;
         const int TA = m * (m + 1) / 2;
         const int TW = Wm != nullptr ? m * (k + 1) : 0;
         const int T = TA + TW;
+        const int Gt = G - cta_first, me = (int)blockIdx.x - cta_first;
+        if (me < 0 || T <= 0) return;
         // tiles are cut into 64 / H row pieces so that a short tile list still spreads over the grid
-        const int lgH = 4 * T <= G ? 4 : (2 * T <= G ? 5 : 6);
+        const int lgH = 4 * T <= Gt ? 4 : (2 * T <= Gt ? 5 : 6);
         const int lgP = 6 - lgH;
         const int TP = T << lgP;
-        struct Piece { double* C; const double* Bsrc; int i0, j0, bcol, tri; };
+        struct Piece { double* C; const double* Bsrc; int i0, j0, tri; };
         auto piece_of = [&](int tp) {
             Piece pc;
             const int t = tp >> lgP;
@@ -399,32 +442,32 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t
                 r = r < 0 ? 0 : (r > m - 1 ? m - 1 : r);
                 while (r > 0 && r * m - r * (r - 1) / 2 > t) --r;
                 while (r + 1 < m && (r + 1) * m - (r + 1) * r / 2 <= t) ++r;
-                const int bi = k + 1 + r, bj = bi + (t - (r * m - r * (r - 1) / 2));
-                pc.C = A; pc.Bsrc = A; pc.i0 = bi * kNB + h0; pc.j0 = bj * kNB; pc.bcol = bj * kNB;
+                const int bi = row_base + r, bj = bi + (t - (r * m - r * (r - 1) / 2));
+                pc.C = A; pc.Bsrc = A; pc.i0 = bi * kNB + h0; pc.j0 = bj * kNB;
                 pc.tri = bi == bj ? h0 : -1;
             } else {
                 const int tw = t - TA;
                 const int r = tw / (k + 1), c = tw - r * (k + 1);
-                pc.C = Wm; pc.Bsrc = Wm; pc.i0 = (k + 1 + r) * kNB + h0; pc.j0 = c * kNB; pc.bcol = c * kNB;
+                pc.C = Wm; pc.Bsrc = Wm; pc.i0 = (row_base + r) * kNB + h0; pc.j0 = c * kNB;
                 pc.tri = -1;
             }
             return pc;
         };
         auto load_piece = [&](const Piece& pc, int stg) {
             double* dst = opnd + stg * 2 * kNB * kCholLd;
-            chol_load_block(dst, A, ld, n, k0, pc.i0, lgH, vec16);                     // U[k0 + kk][i0 + r]
-            chol_load_block(dst + kNB * kCholLd, pc.Bsrc, ld, n, k0, pc.bcol, 6, vec16);   // U or W [k0 + kk][j0 + c]
+            chol_load_block(dst, A, ld, n, k0, pc.i0, lgH, vec16);                      // U[k0 + kk][i0 + r]
+            chol_load_block(dst + kNB * kCholLd, pc.Bsrc, ld, n, k0, pc.j0, 6, vec16);  // U or W [k0 + kk][j0 + c]
         };
         int stage = 0;
         Piece cur{}, nxt{};
-        if ((int)blockIdx.x < TP) {
-            cur = piece_of(blockIdx.x);
+        if (me < TP) {
+            cur = piece_of(me);
             load_piece(cur, 0);
         }
         cp_async_commit();
-        for (int tp = blockIdx.x; tp < TP; tp += G) {
-            if (tp + G < TP) {
-                nxt = piece_of(tp + G);
+        for (int tp = me; tp < TP; tp += Gt) {
+            if (tp + Gt < TP) {
+                nxt = piece_of(tp + Gt);
                 load_piece(nxt, stage ^ 1);
             }
             cp_async_commit();
@@ -440,8 +483,39 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t
             cur = nxt;
         }
         cp_async_wait<0>();
+    };
+
+    strip_phase(0);
+    for (int k = 0; k + 1 < nb; ++k) {
         ++epoch;
         if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
+        // Block row k is final; the updates of block rows < k have been applied everywhere.
+        const int next_items = strip_items(k + 1) > 0 ? strip_items(k + 1) : 1;
+        if (4 * next_items <= G) {
+            // Look-ahead: the first next_items CTAs bring their own strip of block row k + 1 up to date and factorise
+            // it at once, while the other CTAs apply block row k to the rows below k + 1.
+            if ((int)blockIdx.x < next_items) {
+                const int g = blockIdx.x;
+                double* P; int pc0; bool ident;
+                strip_item(k + 1, g, P, pc0, ident);
+                double* ua = opnd + 2 * kNB * kCholLd;        // beyond the strip's own panel buffers
+                double* ub = ua + kNB * kCholLd;
+                const bool need_b = P != nullptr && !ident;
+                __syncthreads();
+                chol_load_block(ua, A, ld, n, k * kNB, (k + 1) * kNB, 6, vec16);
+                if (need_b) chol_load_block(ub, P, ld, n, k * kNB, pc0, 6, vec16);
+                cp_async_commit();
+                chol_strip(A, ld, n, (k + 1) * kNB, P, pc0, ident, g == 0, opnd, vec16, status, ua, need_b ? ub : nullptr);
+                __syncthreads();
+            } else {
+                trailing_phase(k, k + 2, next_items);
+            }
+        } else {
+            trailing_phase(k, k + 1, 0);
+            ++epoch;
+            if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
+            strip_phase(k + 1);
+        }
     }
     cp_async_wait<0>();
     if (tid == 0 && ld_acquire_u32(&bar[1]) != 0u) report(status, PTQ_ERR_TIMEOUT, blockIdx.x, 1);
