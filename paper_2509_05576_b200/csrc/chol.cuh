@@ -96,22 +96,35 @@ __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gsrc, 
 }
 
 // Loads the 64 x ncols block A[r0 .. r0+63][c0 .. c0+ncols-1] into dst[64][kCholLd], ncols = 1 << lg in {16, 32, 64};
-// entries beyond n are zero.
+// entries beyond n are zero.  Every thread copies a fixed column (pair) of successive row groups, so a block that lies
+// inside the matrix needs one pointer increment per copy and no bounds test.
 __device__ __forceinline__ void chol_load_block(double* dst, const double* __restrict__ A, int64_t ld, int n, int r0,
                                                 int c0, int lg, int vec16) {
-    const double* base = A + (int64_t)r0 * ld + c0;
+    const bool interior = r0 + kNB <= n && c0 + (1 << lg) <= n;
     if (vec16) {
         const int sh = lg - 1;                           // pairs per row = 1 << sh
-        for (int idx = threadIdx.x; idx < (kNB << sh); idx += kCholThreads) {
-            const int r = idx >> sh, c = (idx & ((1 << sh) - 1)) * 2;
-            const bool ok = r0 + r < n && c0 + c < n;      // n is even on this path: a pair never straddles n
-            cp_async16_cg(dst + r * kCholLd + c, ok ? base + (int64_t)r * ld + c : A, ok);
+        const int c = (threadIdx.x & ((1 << sh) - 1)) * 2;
+        const int rstep = kCholThreads >> sh;
+        int r = threadIdx.x >> sh;
+        const double* src = A + (int64_t)(r0 + r) * ld + c0 + c;
+        double* d = dst + r * kCholLd + c;
+        if (interior) {
+            for (; r < kNB; r += rstep, src += (int64_t)rstep * ld, d += rstep * kCholLd) cp_async16_cg(d, src, true);
+        } else {
+            for (; r < kNB; r += rstep, src += (int64_t)rstep * ld, d += rstep * kCholLd) {
+                const bool ok = r0 + r < n && c0 + c < n;  // n is even on this path: a pair never straddles n
+                cp_async16_cg(d, ok ? src : A, ok);
+            }
         }
     } else {
-        for (int idx = threadIdx.x; idx < (kNB << lg); idx += kCholThreads) {
-            const int r = idx >> lg, c = idx & ((1 << lg) - 1);
-            const bool ok = r0 + r < n && c0 + c < n;
-            cp_async8(dst + r * kCholLd + c, ok ? base + (int64_t)r * ld + c : A, ok);
+        const int c = threadIdx.x & ((1 << lg) - 1);
+        const int rstep = kCholThreads >> lg;
+        int r = threadIdx.x >> lg;
+        const double* src = A + (int64_t)(r0 + r) * ld + c0 + c;
+        double* d = dst + r * kCholLd + c;
+        for (; r < kNB; r += rstep, src += (int64_t)rstep * ld, d += rstep * kCholLd) {
+            const bool ok = interior || (r0 + r < n && c0 + c < n);
+            cp_async8(d, ok ? src : A, ok);
         }
     }
 }
@@ -241,26 +254,40 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
     const int gc0 = is_diag ? k0 + 16 * warp : pc0 + 16 * (warp - 4);       // first global column of this warp
     const int sc0 = 16 * warp;                                               // first strip column
     double acc[8][2][2];
+    // panel columns that lie inside the matrix and are not the identity: plain vector loads
+    const bool fast_panel = !is_diag && P != nullptr && !identity && vec16 && k0 + kNB <= n && pc0 + kNB <= n;
+    if (fast_panel) {
+        const double* src = P + (int64_t)(k0 + lq) * ld + gc0 + 2 * lr;
 #pragma unroll
-    for (int rb = 0; rb < 8; ++rb)
+        for (int rb = 0; rb < 8; ++rb)
 #pragma unroll
-        for (int cb = 0; cb < 2; ++cb) {
-            const int row = 8 * rb + lq, grow = k0 + row;
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-                const int sc = sc0 + 8 * cb + 2 * lr + e, gc = gc0 + 8 * cb + 2 * lr + e;
-                double val = 0.0;
-                if (is_diag) {
-                    if (sc >= row) {
-                        if (grow < n && gc < n) val = __ldcg(A + (int64_t)grow * ld + gc);
-                        else if (sc == row) val = 1.0;                   // identity padding below n
-                    }
-                } else if (P != nullptr && grow < n && gc < n) {
-                    val = identity ? (sc - kNB == row ? 1.0 : 0.0) : __ldcg(P + (int64_t)grow * ld + gc);
-                }
-                acc[rb][cb][e] = val;
+            for (int cb = 0; cb < 2; ++cb) {
+                const double2 v = __ldcg(reinterpret_cast<const double2*>(src + (int64_t)(8 * rb) * ld + 8 * cb));
+                acc[rb][cb][0] = v.x;
+                acc[rb][cb][1] = v.y;
             }
-        }
+    } else {
+#pragma unroll
+        for (int rb = 0; rb < 8; ++rb)
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                const int row = 8 * rb + lq, grow = k0 + row;
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int sc = sc0 + 8 * cb + 2 * lr + e, gc = gc0 + 8 * cb + 2 * lr + e;
+                    double val = 0.0;
+                    if (is_diag) {
+                        if (sc >= row) {
+                            if (grow < n && gc < n) val = __ldcg(A + (int64_t)grow * ld + gc);
+                            else if (sc == row) val = 1.0;                   // identity padding below n
+                        }
+                    } else if (P != nullptr && grow < n && gc < n) {
+                        val = identity ? (sc - kNB == row ? 1.0 : 0.0) : __ldcg(P + (int64_t)grow * ld + gc);
+                    }
+                    acc[rb][cb][e] = val;
+                }
+            }
+    }
     if (upd_a != nullptr) {
         cp_async_wait<0>();
         __syncthreads();
