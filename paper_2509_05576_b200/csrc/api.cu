@@ -127,6 +127,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(c * c * sizeof(double));
             add(c * c * sizeof(double));
             add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
+            add(chol_scratch_doubles(cols) * sizeof(double));
             break;
         case PTQ_CALL_SENSITIVITY_ORDER:
             if (rows < 1) return 0;
@@ -143,6 +144,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(loss_partials_count(rows, cols) * sizeof(double));
             add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
             add(((size_t)cdiv(rows, kSweepRows) + 1) * sizeof(unsigned));   // per-row-group progress counters of the sweep
+            add(chol_scratch_doubles(cols) * sizeof(double));
             break;
         default:
             return 0;
@@ -190,11 +192,12 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     double* R = cv.take<double>((size_t)n * n);
     double* V = cv.take<double>((size_t)n * n);
     unsigned* bar = cv.take<unsigned>(2);
+    double* Dbuf = cv.take<double>(chol_scratch_doubles(n));
     { Launch l(K_LAMBDA, stream); lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status); }
     { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out); }
     // W = U^-T comes out of the factorisation sweep itself (V must start as zero)
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
-    int st = cholesky_upper(R, n, V, bar, status, stream);
+    int st = cholesky_upper(R, n, V, Dbuf, bar, status, stream);
     if (st) return st;
     st = lauum_lower(V, Hinv, n, stream);
     if (st) return st;
@@ -230,7 +233,7 @@ int ptq_sensitivity_order(const float* W, int rows, int cols, int64_t ldw, const
                                                                               score_mode, partial);
     }
     { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status); }
-    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(S, cols, perm); }
+    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, perm); }
     return launch_status();
 }
 
@@ -255,7 +258,7 @@ int ptq_sensitivity_order_static(const float* W, int rows, int cols, int64_t ldw
                                                                               score_mode, partial);
     }
     { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status); }
-    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(S, cols, perm); }
+    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, perm); }
     return launch_status();
 }
 
@@ -280,6 +283,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     double* partials = cv.take<double>(loss_partials_count(rows, cols));
     unsigned* bar = cv.take<unsigned>(2);
     unsigned* sweep_flags = cv.take<unsigned>((size_t)cdiv(rows, kSweepRows) + 1);
+    double* Dbuf = cv.take<double>(chol_scratch_doubles(n));
 
     // flags and invperm are adjacent pieces of the workspace: clear both
     if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
@@ -288,7 +292,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     { Launch l(K_PERM_CHECK, stream); perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status); }
     { Launch l(K_GATHER_SYM, stream); gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U); }
     { Launch l(K_GATHER_W, stream); gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp); }
-    int st = cholesky_upper(U, n, nullptr, bar, status, stream);   // blocked Eq. 12
+    int st = cholesky_upper(U, n, nullptr, Dbuf, bar, status, stream);   // blocked Eq. 12
     if (st) return st;
 
     st = sweep_launch(Wp, U, E, codes_p, scale, zero, rows, n, bits, sweep_flags, status, stream);
@@ -302,7 +306,10 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
                                                                            zero, codes, What, dW);
     }
     if (want_loss) {
-        GemmParams g = gemm_defaults();     // sum_ij (dW H)_ij dW_ij
+        // sum_ic dW_ic (dW H)_ic; H is symmetric, so for the 64-column block of c only k up to the end of that block is
+        // summed and the blocks before it are doubled
+        GemmParams g = gemm_defaults();
+        g.kend_mode = 1; g.sym_double = 1;
         g.A = dW; g.lda = n; g.a_trans = 0;
         g.B = H_undamped; g.ldb = n; g.b_trans = 0;
         g.M = rows; g.N = n; g.K = n;

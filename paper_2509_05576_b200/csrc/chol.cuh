@@ -237,14 +237,17 @@ __device__ __forceinline__ void chol_strip_blocks(double (&acc)[8][2][2], double
 
 // Factorises the diagonal block of A at k0 and applies the same row operations to 64 panel columns with it: columns
 // pc0 .. pc0 + 63 of rows k0 .. k0 + 63 of the matrix P (row stride ld), or, when `identity` is set, of the identity
-// block (whose transform is the inverse of the transposed diagonal factor).  P == nullptr: diagonal block only.  The
-// diagonal factor is written only when write_diag is set.
+// block (whose transform is the inverse of the transposed diagonal factor).  P == nullptr: diagonal block only.
+// Every CTA working on this block row reads the diagonal block of A, at a time of its own, so the factor of that
+// block is NOT written in place: the CTA with write_diag set stores it to D (64 x 64, row stride 64), and the kernel
+// copies all diagonal factors into A at its very end.
 // When upd_a is given, the strip is first brought up to date with the previous block row (look-ahead):
 //     strip -= upd_a^T [upd_a | upd_b],   upd_a[kk][r] = U[k0 - 64 + kk][k0 + r],  upd_b[kk][c] = P[k0 - 64 + kk][pc0 + c]
 // (both 64 x 64 in shared memory, row stride kCholLd; upd_b == nullptr: the panel part needs no update).
 __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, int n, int k0, double* __restrict__ P,
-                                           int pc0, bool identity, bool write_diag, double* smem, int vec16,
-                                           int32_t* status, const double* upd_a, const double* upd_b) {
+                                           int pc0, bool identity, bool write_diag, double* __restrict__ D,
+                                           double* smem, int vec16, int32_t* status, const double* upd_a,
+                                           const double* upd_b) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int lq = lane >> 2, lr = lane & 3;
     double* Rbuf = smem;
@@ -325,22 +328,30 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
     }
     chol_strip_blocks(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, write_diag && threadIdx.x == 0, status,
                       std::make_integer_sequence<int, 8>());
-    if (is_diag ? write_diag : P != nullptr) {
-        double* M = is_diag ? A : P;
+    if (is_diag) {
+        if (write_diag) {
+#pragma unroll
+            for (int rb = 0; rb < 8; ++rb)
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    const int row = 8 * rb + lq, sc = sc0 + 8 * cb + 2 * lr;
+                    if (sc >= row) D[row * kNB + sc] = acc[rb][cb][0];
+                    if (sc + 1 >= row) D[row * kNB + sc + 1] = acc[rb][cb][1];
+                }
+        }
+    } else if (P != nullptr) {
 #pragma unroll
         for (int rb = 0; rb < 8; ++rb)
 #pragma unroll
             for (int cb = 0; cb < 2; ++cb) {
-                const int row = 8 * rb + lq, grow = k0 + row;
-                const int sc = sc0 + 8 * cb + 2 * lr, gc = gc0 + 8 * cb + 2 * lr;
+                const int grow = k0 + 8 * rb + lq, gc = gc0 + 8 * cb + 2 * lr;
                 if (grow >= n || gc >= n) continue;
-                double* dst = M + (int64_t)grow * ld + gc;
-                const bool keep0 = !is_diag || sc >= row, keep1 = !is_diag || sc + 1 >= row;
-                if (vec16 && keep0) {
+                double* dst = P + (int64_t)grow * ld + gc;
+                if (vec16) {
                     __stcg(reinterpret_cast<double2*>(dst), make_double2(acc[rb][cb][0], acc[rb][cb][1]));
                 } else {
-                    if (keep0) __stcg(dst, acc[rb][cb][0]);
-                    if (keep1 && gc + 1 < n) __stcg(dst + 1, acc[rb][cb][1]);
+                    __stcg(dst, acc[rb][cb][0]);
+                    if (gc + 1 < n) __stcg(dst + 1, acc[rb][cb][1]);
                 }
             }
     }
@@ -412,8 +423,8 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int6
 }
 
 __global__ void __launch_bounds__(kCholThreads, 1)
-chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t ld, int vec16, unsigned* bar,
-                 int32_t* status) {
+chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __restrict__ Dbuf, int n, int64_t ld,
+                 int vec16, unsigned* bar, int32_t* status) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
     int* s_flag = reinterpret_cast<int*>(opnd + 2 * 2 * kNB * kCholLd);     // the strip panels alias opnd
@@ -438,7 +449,8 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t
         for (int g = blockIdx.x; g < reps; g += G) {
             double* P; int pc0; bool ident;
             strip_item(k, g, P, pc0, ident);
-            chol_strip(A, ld, n, k * kNB, P, pc0, ident, g == 0, opnd, vec16, status, nullptr, nullptr);
+            chol_strip(A, ld, n, k * kNB, P, pc0, ident, g == 0, Dbuf + (size_t)k * kNB * kNB, opnd, vec16, status, nullptr,
+                       nullptr);
             __syncthreads();     // the panel buffers are reused by the next repetition and by the trailing phase
         }
     };
@@ -532,7 +544,8 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t
                 chol_load_block(ua, A, ld, n, k * kNB, (k + 1) * kNB, 6, vec16);
                 if (need_b) chol_load_block(ub, P, ld, n, k * kNB, pc0, 6, vec16);
                 cp_async_commit();
-                chol_strip(A, ld, n, (k + 1) * kNB, P, pc0, ident, g == 0, opnd, vec16, status, ua, need_b ? ub : nullptr);
+                chol_strip(A, ld, n, (k + 1) * kNB, P, pc0, ident, g == 0, Dbuf + (size_t)(k + 1) * kNB * kNB, opnd, vec16,
+                           status, ua, need_b ? ub : nullptr);
                 __syncthreads();
             } else {
                 trailing_phase(k, k + 2, next_items);
@@ -545,14 +558,26 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, int n, int64_t
         }
     }
     cp_async_wait<0>();
+    // the diagonal factors move from the side buffer into A once nobody reads the original diagonal blocks any more
+    ++epoch;
+    if (grid_barrier(bar, epoch * (unsigned)G, s_flag)) {
+        for (int b = blockIdx.x; b < nb; b += G)
+            for (int idx = tid; idx < kNB * kNB; idx += kCholThreads) {
+                const int r = idx >> 6, c = idx & 63;
+                if (c >= r && b * kNB + c < n)
+                    A[(int64_t)(b * kNB + r) * ld + b * kNB + c] = __ldcg(Dbuf + (size_t)b * kNB * kNB + idx);
+            }
+    }
     if (tid == 0 && ld_acquire_u32(&bar[1]) != 0u) report(status, PTQ_ERR_TIMEOUT, blockIdx.x, 1);
 }
 
 // In-place blocked upper Cholesky A = U^T U of the n x n matrix A (row stride n).  Only the upper triangle is read or
 // written.  With Wm (n x n, zero on entry) the same sweep also leaves W = U^-T there (lower triangular): the row
 // operations of the factorisation are applied to the identity, Sec. 5 item 1's "inverse of the decomposed result".
-// `bar` is 2 x uint32 of device scratch.
-inline int cholesky_upper(double* A, int n, double* Wm, unsigned* bar, int32_t* status, cudaStream_t stream) {
+// `bar` is 2 x uint32 of device scratch, Dbuf holds chol_scratch_doubles(n) doubles (the diagonal factors on their way).
+inline size_t chol_scratch_doubles(int n) { return (size_t)((n + kNB - 1) / kNB) * kNB * kNB; }
+inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* bar, int32_t* status,
+                          cudaStream_t stream) {
     static int grid = 0;
     if (grid == 0) {
         if (cudaFuncSetAttribute(chol_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -571,7 +596,7 @@ inline int cholesky_upper(double* A, int n, double* Wm, unsigned* bar, int32_t* 
     if (cudaMemsetAsync(bar, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int64_t ld = n;
     int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;
-    void* args[] = {&A, &Wm, &n, &ld, &vec16, &bar, &status};
+    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status};
     Launch l(K_CHOL_COOP, stream);
     if (cudaLaunchCooperativeKernel((const void*)chol_coop_kernel, dim3(grid), dim3(kCholThreads), args,
                                     kCholSmemBytes, stream) != cudaSuccess) {

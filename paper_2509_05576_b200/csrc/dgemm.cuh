@@ -18,6 +18,8 @@ struct GemmParams {
     double alpha, beta;
     int kbeg_mode;     // 0: k from 0;  1: from max(i0, j0);  2: from i0   (operands are zero before that)
     int kend_mode;     // 0: k to K;    1: to min(K, j0 + BN)              (B is zero after that)
+    int sym_double;    // B symmetric, C not written (reduction epilogue): with kend_mode 1, the k blocks before the tile's
+                       // own column block count twice, which stands in for the skipped blocks after it
     int upper_only;    // skip tiles that lie entirely below the diagonal
     int mirror;        // also store C[j][i] for tiles above the diagonal
     // batch z = blockIdx.z: operands advance by these element strides
@@ -55,9 +57,10 @@ __device__ __forceinline__ void dmma_884(double& c0, double& c1, double a, doubl
                  : "d"(a), "d"(b));
 }
 
-// BT x BT output tile, 256 threads = 8 warps as 2 x 4; each warp owns (BT/2) x (BT/4) outputs as 8 x 8 fragments.
+// BT x BT output tile (bx, by) of batch z, 256 threads = 8 warps as 2 x 4; each warp owns (BT/2) x (BT/4) outputs as
+// 8 x 8 fragments.  nbx = number of column tiles (indexes the partials).
 template <int BT>
-__global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
+__device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, int z, int nbx, int nby) {
     constexpr int BK = kGemmBK;
     constexpr int LDM = BT + 4;            // row stride of an m-contiguous operand tile
     constexpr int TILE = BT * kGemmLdk;
@@ -66,7 +69,6 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
     constexpr int EPT = BT * BK / kGemmThreads;
     extern __shared__ __align__(16) double smem[];
 
-    const int z = blockIdx.z;
     int N = p.N, K = p.K;
     if (p.ragN_step > 0) {
         int lim = p.ragN_lim - z * p.ragN_step;
@@ -75,7 +77,7 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
     }
     if (p.k_is_n) K = N;
     const int M = p.M;
-    const int i0 = blockIdx.y * BT, j0 = blockIdx.x * BT;
+    const int i0 = by * BT, j0 = bx * BT;
     if (i0 >= M || j0 >= N) return;
     if (p.upper_only && i0 >= j0 + BT) return;
 
@@ -141,6 +143,12 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
     for (int kt = 0; kt < nkt; ++kt) {
         cp_async_wait<kGemmStages - 2>();
         __syncthreads();
+        if (p.sym_double && kbeg + kt * BK == j0) {
+#pragma unroll
+            for (int a = 0; a < FM; ++a)
+#pragma unroll
+                for (int b = 0; b < FN; ++b) { acc[a][b][0] *= 2.0; acc[a][b][1] *= 2.0; }
+        }
         if (kt + kGemmStages - 1 < nkt) load_stage((kt + kGemmStages - 1) % kGemmStages, kbeg + (kt + kGemmStages - 1) * BK);
         cp_async_commit();
         const double* as = smem + (size_t)(kt % kGemmStages) * 2 * TILE;
@@ -182,7 +190,8 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
             __syncthreads();
         }
         if (tid == 0)
-            p.partials[((int64_t)z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x] = red[0];
+            p.partials[((int64_t)z * nby + by) * nbx + bx] = red[0];
+        __syncthreads();
         return;
     }
 
@@ -203,6 +212,23 @@ __global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
                 if (do_mirror) C[(int64_t)gj * p.ldc + gi] = v;
             }
     }
+}
+
+// With sym_double the grid has half as many column tiles: CTA x handles column tiles x and nbx - 1 - x, whose k ranges
+// (64 (x + 1) and 64 (nbx - x)) add up to the same length for every CTA.
+template <int BT>
+__global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
+    if (p.sym_double) {
+        const int nbx = (p.N + BT - 1) / BT;
+        const int bx = blockIdx.x, bx2 = nbx - 1 - bx;
+        dgemm_tile<BT>(p, bx, blockIdx.y, blockIdx.z, nbx, gridDim.y);
+        if (bx2 > bx) {
+            __syncthreads();
+            dgemm_tile<BT>(p, bx2, blockIdx.y, blockIdx.z, nbx, gridDim.y);
+        }
+        return;
+    }
+    dgemm_tile<BT>(p, blockIdx.x, blockIdx.y, blockIdx.z, gridDim.x, gridDim.y);
 }
 
 inline GemmParams gemm_defaults() {
@@ -230,7 +256,8 @@ inline int launch_dgemm(int kernel_id, const GemmParams& p, int batches, cudaStr
         bt = tiles128 >= 2 * 148 ? 128 : 64;
     }
     dim3 grid(cdiv(p.N, bt), cdiv(p.M, bt), batches);
-    if (grid_out) *grid_out = grid;
+    if (grid_out) *grid_out = grid;          // the tile grid (what the partials are indexed by)
+    if (p.sym_double) grid.x = (grid.x + 1) / 2;
     Launch scope(kernel_id, stream);
     if (bt == 128)
         dgemm_kernel<128><<<grid, kGemmThreads, gemm_smem_bytes<128>(), stream>>>(p);

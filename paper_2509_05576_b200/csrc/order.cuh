@@ -105,24 +105,29 @@ __device__ __forceinline__ unsigned long long sortable_key(double x) {
 }
 
 // perm[rank_j] = j with rank_j = #{k : S_k > S_j, or S_k == S_j and k < j}: a stable descending sort by counting.
+// 32 columns j per CTA; the eight lanes that share a column each count a strided eighth of the keys.
+constexpr int kRankCols = 32;
 __global__ void __launch_bounds__(256) rank_sort_kernel(const double* __restrict__ S, int cols,
                                                          int32_t* __restrict__ perm) {
-    __shared__ unsigned long long keys[256];
-    const int j = blockIdx.x * 256 + threadIdx.x;
+    __shared__ unsigned long long keys[1024];
+    const int j = blockIdx.x * kRankCols + (threadIdx.x >> 3);
+    const int part = threadIdx.x & 7;
     const unsigned long long kj = j < cols ? sortable_key(S[j]) : 0ull;
     int rank = 0;
-    for (int t0 = 0; t0 < cols; t0 += 256) {
-        const int k = t0 + threadIdx.x;
-        keys[threadIdx.x] = k < cols ? sortable_key(S[k]) : 0ull;
+    for (int t0 = 0; t0 < cols; t0 += 1024) {
+        for (int t = threadIdx.x; t < 1024; t += 256) keys[t] = t0 + t < cols ? sortable_key(S[t0 + t]) : 0ull;
         __syncthreads();
-        const int lim = min(256, cols - t0);
-        for (int t = 0; t < lim; ++t) {
+        const int lim = min(1024, cols - t0);
+        for (int t = part; t < lim; t += 8) {
             const unsigned long long kk = keys[t];
             rank += (kk > kj || (kk == kj && (t0 + t) < j)) ? 1 : 0;
         }
         __syncthreads();
     }
-    if (j < cols) perm[rank] = j;
+    rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+    rank += __shfl_xor_sync(0xffffffffu, rank, 2);
+    rank += __shfl_xor_sync(0xffffffffu, rank, 4);
+    if (part == 0 && j < cols) perm[rank] = j;
 }
 
 }  // namespace ptq

@@ -44,7 +44,7 @@ def test_workspace_sizes(lib):
         assert 0 < small < big
         assert small % 256 == 0
     # the inverse needs two cols x cols float64 matrices
-    assert 2 * 2304 * 2304 * 8 <= ptq.workspace_bytes(ptq.CALL_PREPARE_HINV, 0, 2304, 0) <= 2 * 2304 * 2304 * 8 + 4096
+    assert 2 * 2304 * 2304 * 8 <= ptq.workspace_bytes(ptq.CALL_PREPARE_HINV, 0, 2304, 0) <= 2 * 2304 * 2304 * 8 + 2304 * 64 * 8 + 4096
     assert ptq.workspace_bytes(99, 1, 1, 1) == 0
     # largest benchmark shape stays far below the 180 GB of one GPU
     total = sum(ptq.workspace_bytes(c, 4096, 11008, 8192) for c in range(4))

@@ -101,3 +101,41 @@ def test_resnet50_512x4608_cols_exceed_calibration_columns():
 def test_yolov5s_extra_512x4608_8bit():
     spec = _find(wl.config4(bits=(8,)), "y512x4608")
     assert _row_subset_parity(spec, 32, seed=2) == 0
+
+
+def test_more_block_rows_than_sms():
+    """9600 columns = 150 block rows of 64, more than the 148 CTAs of the persistent factorisation kernel, so its strip
+    work wraps around the grid.  The CPU oracle is out of reach at this width (cols^3 work), so the checks are the
+    defining properties: Hinv (H + lambda I) = I, the status word, and the loss against its definition."""
+    rows, cols, n, bits = 40, 9600, 1024, 4
+    spec = wl.LayerSpec("wide", rows, cols, n, bits, "kaiming", "normal", 77)
+    W, X = wl.make_layer(spec)
+    bufs = ptq.quantize_layer_full(torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda(), bits, spec.damp)
+    torch.cuda.synchronize()
+    ptq.check_status(bufs.status, "wide layer")
+    H, Hinv = bufs.H, bufs.Hinv
+    Xd = torch.from_numpy(X).cuda().double()
+    rs = slice(0, cols, 37)                                              # a spread of rows
+    assert float((H[rs] - 2.0 * (Xd[rs] @ Xd.T)).abs().max()) <= 1e-11 * float(H.abs().max())
+    Hd = H + bufs.lam * torch.eye(cols, dtype=torch.float64, device="cuda")
+    R = Hinv[rs] @ Hd
+    R -= torch.eye(cols, dtype=torch.float64, device="cuda")[rs]
+    assert float(R.abs().max()) <= 1e-9
+    assert torch.equal(Hinv, Hinv.T)
+    perm = bufs.perm.cpu().numpy()
+    assert sorted(perm.tolist()) == list(range(cols))
+    S = bufs.S.cpu().numpy()
+    assert np.all(np.diff(S[perm]) <= 0)
+    codes = bufs.codes.cpu().numpy()
+    assert codes.max() <= 2 ** bits - 1
+    What = bufs.What.double()
+    sc, zp = bufs.scale.double(), bufs.zero.double()
+    assert torch.equal(What.float(), (sc[:, None] * (bufs.codes.double() - zp[:, None])).float())
+    dW = torch.from_numpy(W).cuda().double() - What
+    loss_def = 0.5 * float(((dW @ H) * dW).sum())
+    assert abs(float(bufs.loss.item()) - loss_def) <= 1e-9 * loss_def
+    # the compensated result must beat plain round-to-nearest on the same grid
+    Wd = torch.from_numpy(W).cuda().double()
+    rtn = sc[:, None] * (torch.clamp(torch.round(Wd / sc[:, None]) + zp[:, None], 0, 2 ** bits - 1) - zp[:, None])
+    dR = Wd - rtn.float().double()
+    assert loss_def < 0.5 * float(((dR @ H) * dR).sum())
