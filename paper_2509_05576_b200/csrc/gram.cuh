@@ -13,7 +13,8 @@
 // streams 64-wide K blocks of all six slices of the 128 "row" columns and of the 64 "column" columns
 // (SWIZZLE_64B, 3 stages of 72 KB); one thread issues the 42 tcgen05.mma.kind::i8 instructions of a stage into six
 // TMEM accumulators (6 x 64 columns); four epilogue warps read the accumulators back with tcgen05.ld, combine the
-// groups exactly in int64, scale by 2^(41 - sh_i - sh_j) and add into H.
+// groups exactly in int64, hand TMEM back (the next tile's products then overlap the rest of the epilogue), scale by
+// 2^(41 - sh_i - sh_j) and add into H.
 // Every wait on an mbarrier is bounded; when one expires the CTA records PTQ_ERR_TIMEOUT, drains and returns.
 #pragma once
 #include <cuda.h>
@@ -192,6 +193,22 @@ __device__ __forceinline__ uint64_t make_desc_sw64(uint32_t smem_addr) {
     return d;
 }
 
+// The same descriptor as two 32-bit words; the address field (bits 0..13, shared-memory address / 16) is added to the
+// low word at run time: all tiles lie below 256 KB, so the sum never leaves the field.
+constexpr uint32_t kDescLo = 1u << 16;
+constexpr uint32_t kDescHi = (uint32_t)(512 >> 4) | (1u << 14) | (4u << 29);
+__device__ __forceinline__ void tc_mma_i8_lohi(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t hi,
+                                               uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, {%6, %6, %6, %6}, p;\n\t}\n"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(accumulate), "r"(0u)
+        : "memory");
+}
+
 // Instruction descriptor: int8 x int8 -> int32, both operands K-major, M = 128, N = 64.
 constexpr uint32_t kGramIdesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kGramTN >> 3) << 17) |
                                 ((uint32_t)(kGramTM >> 4) << 24);
@@ -299,19 +316,22 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                     ok = mbar_wait_bounded(full_bar(stage), phase, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sbase = base + stage * kGramStageBytes;
+                    // Descriptors: A and B tiles share the high word; the low word is the stage's address field plus a
+                    // compile-time offset per slice and per 32-byte K step, so each MMA costs two integer adds.
+                    const uint32_t sb = kDescLo + ((base + stage * kGramStageBytes) >> 4);
+                    const uint32_t first = kb > 0 ? 1u : 0u;      // the first product of a group overwrites on kb == 0
 #pragma unroll
                     for (int t = 0; t < kGroups; ++t) {
 #pragma unroll
                         for (int a = 0; a <= t; ++a) {
                             const int b = t - a;
-                            const uint64_t ad = make_desc_sw64(sbase + a * kGramABytes);
-                            const uint64_t bd = make_desc_sw64(sbase + kSlices * kGramABytes + b * kGramBBytes);
 #pragma unroll
                             for (int ks = 0; ks < kGramKB / 32; ++ks) {
-                                const uint32_t acc = (kb > 0 || a > 0 || ks > 0) ? 1u : 0u;
-                                tc_mma_i8(tmem_base + t * kGramTN, ad + (uint64_t)(ks * 2), bd + (uint64_t)(ks * 2),
-                                          kGramIdesc, acc);
+                                const uint32_t alo = sb + (uint32_t)((a * kGramABytes) >> 4) + (uint32_t)(ks * 2);
+                                const uint32_t blo = sb + (uint32_t)((kSlices * kGramABytes + b * kGramBBytes) >> 4) +
+                                                     (uint32_t)(ks * 2);
+                                tc_mma_i8_lohi(tmem_base + t * kGramTN, alo, blo, kDescHi, kGramIdesc,
+                                               (a > 0 || ks > 0) ? 1u : first);
                             }
                         }
                     }
@@ -336,7 +356,10 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             tc_fence_after();
             const int row = bi * kGramTM + r_in_tile;
             const int sh_i = row < cols ? shifts[row] : 0;
-#pragma unroll 1
+            // 1. drain the accumulators into registers: v = G0 2^40 + G1 2^32 + ... + G5, combined exactly in int64 and
+            //    rounded once to float64; then TMEM is handed back, so that the next tile's products run under step 2
+            double v[kGramTN];
+#pragma unroll
             for (int ch = 0; ch < kGramTN / 16; ++ch) {
                 long long lo[16], hi[16];
                 uint32_t r[16];
@@ -360,26 +383,34 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_ld16(taddr + 0 * kGramTN, r); tc_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 16; ++c) hi[c] += (long long)(int)r[c] << 16;
-                if (row < cols) {
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const int col = bj * kGramTN + ch * 16 + c;
-                        if (col < cols) {
-                            const double v = fma((double)hi[c], 16777216.0, (double)lo[c]);
-                            const int e = 41 - sh_i - shifts[col];
-                            const double add = scalbn(v, e);
-                            // tiles that straddle the diagonal hold both (i, j) and (j, i): each writes itself only
-                            const bool straddle = (bj * kGramTN < bi * kGramTM + kGramTM);
-                            const double out = H[(int64_t)row * cols + col] + add;
-                            H[(int64_t)row * cols + col] = out;
-                            if (!straddle) H[(int64_t)col * cols + row] = out;
-                        }
-                    }
-                }
+                for (int c = 0; c < 16; ++c) v[ch * 16 + c] = fma((double)hi[c], 16777216.0, (double)lo[c]);
             }
             tc_fence_before();
             mbar_arrive(acc_empty);
             acc_phase ^= 1u;
+            // 2. H += v 2^(41 - sh_i - sh_j).  Tiles away from the diagonal also own the mirrored entries (j, i); since H
+            //    is symmetric the old value is read there, where consecutive lanes (rows i) are contiguous.
+            if (row < cols) {
+                const bool straddle = (bj * kGramTN < bi * kGramTM + kGramTM);
+                const double fi = __longlong_as_double((long long)(1023 + 20 - sh_i) << 52);     // 2^(20 - sh_i)
+#pragma unroll
+                for (int c = 0; c < kGramTN; ++c) {
+                    const int col = bj * kGramTN + c;
+                    if (col < cols) {
+                        const double fj = __longlong_as_double((long long)(1023 + 21 - shifts[col]) << 52);
+                        const double add = (v[c] * fi) * fj;                // exact: powers of two, no under/overflow
+                        if (straddle) {
+                            // tiles that straddle the diagonal hold both (i, j) and (j, i): each writes itself only
+                            H[(int64_t)row * cols + col] += add;
+                        } else {
+                            const double out = H[(int64_t)col * cols + row] + add;
+                            H[(int64_t)col * cols + row] = out;
+                            H[(int64_t)row * cols + col] = out;
+                        }
+                    }
+                }
+            }
         }
     }
 
