@@ -50,7 +50,8 @@ __global__ void gather_w_kernel(const float* __restrict__ W, int rows, int cols,
 // Rows never interact (Sec. 4.2 step 4: every row of the current column is quantized at once, independently), so
 // the rows are cut into groups of 32 and each group is an independent pipeline.  A group is served by `cpg` CTAs;
 // the 64-column blocks are dealt to them round-robin (CTA i owns blocks i, i + cpg, ...).  The owner of block b
-// quantizes it, writes the scaled errors E[:, b] and the codes, and raises the group's counter to b + 1.  Every CTA
+// quantizes it, writes the scaled errors E[:, b] and the codes, eight columns at a time, and raises the group's counter
+// with every piece (8 b + 8 once the block is complete).  Every CTA
 // of the group then applies E[:, b] to the blocks IT owns: W[:, b'] -= E[:, b] U[b, b'] (the deferred part of Eq. 11),
 // a 32 x 64 x 64 float64 tensor-core MMA tile per block.  All updates of one block are made by its owner, in order, so
 // no block is ever touched by two CTAs; the only cross-CTA dependency is "E[:, b] is ready".  The owner of block b + 1
@@ -63,15 +64,14 @@ __global__ void gather_w_kernel(const float* __restrict__ W, int rows, int cols,
 //         c = clamp(rint(w / s) + z),  d = w - q,  w_j -= d U[p][j] / U[p][p]   (j inside the mini-block),
 //     with warp-private shared-memory staging only, then publishes the 32 x 8 differences d;
 //   - the warps to its right subtract d (U[p][j] / U[p][p]) from their fragments: a rank-8 update, two MMAs per
-//     fragment.  One block-wide barrier per mini-block.
+//     fragment.  One barrier per mini-block, among the warps from m rightwards only.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kSweepThreads = 256;
 constexpr int kSweepRows = 32;
 constexpr int kSweepLd = kNB + 4;                                   // 68: conflict-free MMA operand stride
-constexpr int kSweepEsLd = kNB + 1;                                 // 65: row-per-lane writes of E
 constexpr int kSweepTLd = 9;                                        // fragment <-> row-per-lane staging
 constexpr int kSweepDLd = 12;                                       // 32 x 8 differences as MMA operand A
-constexpr int kSweepSmemDoubles = kNB * kSweepLd /*Us*/ + kNB /*rdiag*/ + kSweepRows * kSweepEsLd /*Es*/ +
+constexpr int kSweepSmemDoubles = kNB * kSweepLd /*Us*/ + kNB /*rdiag*/ +
                                   kSweepRows * kSweepTLd /*T*/ + 2 * kSweepRows * kSweepDLd /*Dm*/ +
                                   kSweepRows * kSweepLd /*Ea*/ + 2 * kNB * kSweepLd /*Bb*/;
 constexpr size_t kSweepSmemBytes = sizeof(double) * kSweepSmemDoubles + kSweepRows * (kNB + 4) + 16;
@@ -84,7 +84,7 @@ struct SweepParams {
     const float* scale;
     const float* zero;
     int rows, n, bits, vec16;
-    unsigned* flags;        // [groups] finished blocks per group, then [1] abort word; zero at launch
+    unsigned* flags;        // [groups] published 8-column pieces of E per group, then [1] abort word; zero at launch
     int32_t* status;
 };
 
@@ -150,8 +150,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
     extern __shared__ __align__(16) unsigned char sweep_smem[];
     double* Us = reinterpret_cast<double*>(sweep_smem);                // [64][68] diagonal block of U, rows / pivot
     double* rdiag = Us + kNB * kSweepLd;                               // [64] 1 / U_pp
-    double* Es = rdiag + kNB;                                          // [32][65] scaled errors of the block
-    double* T = Es + kSweepRows * kSweepEsLd;                          // [32][9] staging of the current mini-block
+    double* T = rdiag + kNB;                          // [32][9] staging of the current mini-block
     double* Dm = T + kSweepRows * kSweepTLd;                           // [2][32][12] differences of a mini-block
     double* Ea = Dm + 2 * kSweepRows * kSweepDLd;                      // [32][68] MMA operand A: E[:, e]
     double* Bb = Ea + kSweepRows * kSweepLd;                           // [2][64][68] MMA operand B: U[e, b']
@@ -197,6 +196,15 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 
     for (int g = g_first; g < groups; g += g_step) {
         const int r0 = g * kSweepRows;
+        // the grid of this lane's row (one row per lane in the chains), fixed for the whole group
+        const int row = r0 + lane;
+        const bool live = row < rows;
+        RowGrid rg;
+        rg.sc = live ? (double)prm.scale[row] : 1.0;
+        rg.zp = live ? (double)prm.zero[row] : 0.0;
+        rg.rsc = 1.0 / rg.sc;
+        rg.lo = -rg.zp;
+        rg.hi = maxq - rg.zp;
         int lazy = 0;
         bool prepared = false;           // Us / rdiag / blk already hold the block about to be quantized
         // the block being quantized: fragment a = rows 8 a + lq, columns 8 warp + 2 lr + {0, 1}
@@ -227,17 +235,11 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         }
                 }
                 __syncthreads();
-                const int row = r0 + lane;
-                const bool live = row < rows;
-                RowGrid rg;
-                rg.sc = live ? (double)prm.scale[row] : 1.0;
-                rg.zp = live ? (double)prm.zero[row] : 0.0;
-                rg.rsc = 1.0 / rg.sc;
-                rg.lo = -rg.zp;
-                rg.hi = maxq - rg.zp;
 #pragma unroll
                 for (int m = 0; m < 8; ++m) {
                     double* dm = Dm + (m & 1) * kSweepRows * kSweepDLd;
+                    double v[8];
+                    if (warp < m) continue;          // this warp's columns are done; it is out of the remaining barriers
                     if (warp == m) {
                         // fragments -> one row per lane
 #pragma unroll
@@ -245,7 +247,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 #pragma unroll
                             for (int e = 0; e < 2; ++e) T[(8 * a + lq) * kSweepTLd + 2 * lr + e] = blk[a][e];
                         __syncwarp();
-                        double v[8], lev[8];
+                        double lev[8];
 #pragma unroll
                         for (int c = 0; c < 8; ++c) v[c] = T[lane * kSweepTLd + c];
                         const double* us = Us + (8 * m) * kSweepLd + 8 * m;
@@ -258,13 +260,35 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             dm[lane * kSweepDLd + c] = v[c];
-                            Es[lane * kSweepEsLd + 8 * m + c] = v[c] * rdiag[8 * m + c];
                             Cs[lane * (kNB + 4) + 8 * m + c] = (uint8_t)(int)(lev[c] + rg.zp);
                         }
                     }
-                    if (m == 7) break;
-                    __syncthreads();
-                    if (warp > m) {
+                    // the differences of mini-block m become visible to the warps right of it (only those take part)
+                    if (m < 7) asm volatile("bar.sync 1, %0;" ::"r"((8 - m) * 32) : "memory");
+                    if (warp == m) {
+                        // The scaled errors e = d / U_pp of these eight columns go out at once, off the critical path
+                        // (the warps to the right are already updating): the owner of the next block folds them into its
+                        // block while the rest of this block is still being quantized.
+                        if (live) {
+                            double* dst = prm.E + (int64_t)row * n + p0 + 8 * m;
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) v[c] *= rdiag[8 * m + c];
+                            if (prm.vec16 && p0 + 8 * m + 8 <= n) {
+#pragma unroll
+                                for (int c = 0; c < 8; c += 2)
+                                    __stcg(reinterpret_cast<double2*>(dst + c), make_double2(v[c], v[c + 1]));
+                            } else {
+#pragma unroll
+                                for (int c = 0; c < 8; ++c)
+                                    if (p0 + 8 * m + c < n) __stcg(dst + c, v[c]);
+                            }
+                        }
+                        if (cpg > 1) {
+                            __threadfence();
+                            __syncwarp();
+                            if (lane == 0) atomicExch(&prm.flags[g], (unsigned)(8 * b + m + 1));
+                        }
+                    } else {
                         // rank-8 update of this warp's columns: blk -= d (U'[8 m .. 8 m + 7][8 warp .. 8 warp + 7])
                         const double b0 = Us[(8 * m + lr) * kSweepLd + 8 * warp + lq];
                         const double b1 = Us[(8 * m + 4 + lr) * kSweepLd + 8 * warp + lq];
@@ -280,27 +304,16 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                 __syncthreads();
                 for (int idx = tid; idx < kSweepRows * kNB; idx += kSweepThreads) {
                     const int r = idx >> 6, c = idx & 63;
-                    if (r0 + r < rows && c < kb) __stcg(prm.E + (int64_t)(r0 + r) * n + p0 + c, Es[r * kSweepEsLd + c]);
-                }
-                if (cpg > 1) {
-                    __syncthreads();
-                    if (tid == 0) {
-                        __threadfence();
-                        atomicExch(&prm.flags[g], (unsigned)(b + 1));
-                    }
-                }
-                for (int idx = tid; idx < kSweepRows * kNB; idx += kSweepThreads) {
-                    const int r = idx >> 6, c = idx & 63;
                     if (r0 + r < rows && c < kb) prm.codes_p[(int64_t)(r0 + r) * n + p0 + c] = Cs[r * (kNB + 4) + c];
                 }
                 prepared = false;
-            } else {
-                // ------------------------------------------------------------ wait for E[:, b]
+            } else if (!next_mine) {
+                // ------------------------------------------------------------ wait for all of E[:, b]
                 if (tid == 0) {
                     const long long t0 = clock64();
                     int ok = 1;
                     unsigned it = 0;
-                    while (ld_acquire_u32(&prm.flags[g]) < (unsigned)(b + 1)) {
+                    while (ld_acquire_u32(&prm.flags[g]) < (unsigned)(8 * (b + 1))) {
                         if ((++it & 63u) == 0u) {
                             if (ld_acquire_u32(abort_word) != 0u) { ok = 0; break; }
                             if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); ok = 0; break; }
@@ -320,8 +333,6 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
             // ---------------------------------------------------------------- deferred Eq. 11 on the owned blocks
             if (next_mine) {
                 // block b + 1 only, straight into the fragments the chain starts from; the other blocks catch up later
-                sweep_load_tile(Ea, kSweepLd, prm.E, n, r0, p0, kSweepRows, kNB, rows, n, prm.vec16);
-                cp_async_commit();
 #pragma unroll
                 for (int a = 0; a < 4; ++a)
 #pragma unroll
@@ -330,18 +341,54 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
                     }
                 cp_async_wait<0>();
-                __syncthreads();
-                double prod[4][2];
+                __syncthreads();             // U[b, b + 1] is in Bb
+                // E[:, b] arrives eight columns at a time.  Every warp polls the group's counter for itself (bounded),
+                // requests the operand of piece m straight from global memory as soon as it is out, and meanwhile
+                // multiplies piece m - 1, whose operand was requested one piece earlier.
+                double prod[4][2], af[2][2][4];        // af[piece parity][k step][row fragment]
 #pragma unroll
                 for (int a = 0; a < 4; ++a) prod[a][0] = prod[a][1] = 0.0;
-#pragma unroll 4
-                for (int kk = 0; kk < kNB; kk += 4) {
-                    const double bf = Bb[(kk + lr) * kSweepLd + 8 * warp + lq];
+                bool ok = true;
+                unsigned seen = 0;
 #pragma unroll
-                    for (int a = 0; a < 4; ++a) {
-                        const double af = Ea[(8 * a + lq) * kSweepLd + kk + lr];
-                        dmma_884(prod[a][0], prod[a][1], af, bf);
+                for (int m = 0; m <= 8; ++m) {
+                    if (m < 8) {
+                        if (seen < (unsigned)(8 * b + m + 1)) {      // poll only when the last look was not enough
+                            if (lane == 0) {
+                                const long long t0 = clock64();
+                                unsigned it = 0;
+                                while ((seen = ld_acquire_u32(&prm.flags[g])) < (unsigned)(8 * b + m + 1)) {
+                                    if ((++it & 63u) == 0u) {
+                                        if (ld_acquire_u32(abort_word) != 0u) { ok = false; break; }
+                                        if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); ok = false; break; }
+                                    }
+                                }
+                                __threadfence();
+                            }
+                            seen = __shfl_sync(0xffffffffu, seen, 0);
+                            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                            if (!ok) break;
+                        }
+#pragma unroll
+                        for (int s4 = 0; s4 < 2; ++s4)
+#pragma unroll
+                            for (int a = 0; a < 4; ++a) {
+                                const int r = r0 + 8 * a + lq;
+                                af[m & 1][s4][a] = r < rows ? __ldcg(prm.E + (int64_t)r * n + p0 + 8 * m + 4 * s4 + lr) : 0.0;
+                            }
                     }
+                    if (m > 0) {
+#pragma unroll
+                        for (int s4 = 0; s4 < 2; ++s4) {
+                            const double bf = Bb[(8 * (m - 1) + 4 * s4 + lr) * kSweepLd + 8 * warp + lq];
+#pragma unroll
+                            for (int a = 0; a < 4; ++a) dmma_884(prod[a][0], prod[a][1], af[(m - 1) & 1][s4][a], bf);
+                        }
+                    }
+                }
+                if (__syncthreads_or(ok ? 0 : 1)) {
+                    if (tid == 0) report(prm.status, PTQ_ERR_TIMEOUT, blockIdx.x, 3);
+                    return;
                 }
 #pragma unroll
                 for (int a = 0; a < 4; ++a) {
