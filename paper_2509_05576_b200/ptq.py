@@ -275,3 +275,55 @@ def quantize_layer_full(W, X, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG, sco
                                               bufs.What, bufs.H if want_loss else None,
                                               bufs.loss if want_loss else None, ws, st, s))
     return bufs
+
+
+class HostStaging:
+    """Device landing buffers and the copy stream used by ``quantize_layer_from_host`` (allocated once per shape)."""
+
+    def __init__(self, rows, cols, chunk_cols, device="cuda"):
+        d = torch.device(device)
+        self.W = torch.empty((rows, cols), dtype=torch.float32, device=d)
+        self.X = [torch.empty((cols, nc), dtype=torch.float32, device=d) for nc in chunk_cols]
+        self.copy_stream = torch.cuda.Stream(device=d)
+
+
+def quantize_layer_from_host(W_host, X_batches_host, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG,
+                             score_mode=SCORE_QERR, bufs=None, ws=None, staging=None, stream=None, want_loss=True):
+    """The whole path for a layer whose W and calibration activations sit in (pinned) host memory.
+
+    ``X_batches_host`` is a list of contiguous [cols, n_i] float32 tensors, the calibration batches.  They are uploaded
+    one after the other on a copy stream while the Hessian of the batches already on the device is being accumulated
+    (``ptq_hessian_accumulate`` is additive over calibration columns), so most of the upload hides behind the Gram.
+    Everything is asynchronous; returns the LayerBuffers (outputs on the device).
+    """
+    rows, cols = W_host.shape
+    staging = staging or HostStaging(rows, cols, [x.shape[1] for x in X_batches_host])
+    bufs = bufs or LayerBuffers(rows, cols)
+    ws = ws or Workspace()
+    s = torch.cuda.current_stream() if stream is None else stream
+    cs = staging.copy_stream
+    st = bufs.status
+    cs.wait_stream(s)                       # the landing buffers are free once earlier work on the stream is done
+    events = []
+    with torch.cuda.stream(cs):
+        for xd, xh in zip(staging.X, X_batches_host):
+            xd.copy_(xh, non_blocking=True)
+            ev = torch.cuda.Event()
+            ev.record(cs)
+            events.append(ev)
+        staging.W.copy_(W_host, non_blocking=True)
+        w_ready = torch.cuda.Event()
+        w_ready.record(cs)
+    with torch.cuda.stream(s):
+        st.zero_()
+        bufs.H.zero_()
+        for xd, ev in zip(staging.X, events):
+            s.wait_event(ev)
+            hessian_accumulate(bufs.H, xd, ws, st, s)
+        prepare_hinv(bufs.H, damp, damp_mode, bufs.Hinv, bufs.Hinv_diag, bufs.lam, ws, st, s)
+        s.wait_event(w_ready)
+        minmax_grid(staging.W, bits, bufs.scale, bufs.zero, st, s)
+        sensitivity_order(staging.W, bufs.Hinv_diag, bufs.scale, bufs.zero, bits, score_mode, bufs.S, bufs.perm, ws, st, s)
+        quantize_layer(staging.W, bufs.Hinv, bufs.perm, bufs.scale, bufs.zero, bits, bufs.codes, bufs.What,
+                       bufs.H if want_loss else None, bufs.loss if want_loss else None, ws, st, s)
+    return bufs
