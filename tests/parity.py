@@ -6,7 +6,7 @@ import torch
 import oracle
 from paper_2509_05576_b200 import ptq
 
-# Tolerances (the acceptance rule of the task): column order and integer codes bit-exact, except that codes whose
+# Tolerances: column order and integer codes bit-exact, except that codes whose
 # pre-rounding value lies within 1e-4 (in units of the row's scale) of a rounding boundary may differ by one level on
 # at most 0.1 % of the weights; dequantized weights within 1e-4 relative; reconstruction loss within 1e-3 relative.
 BOUNDARY_TOL = 1e-4
