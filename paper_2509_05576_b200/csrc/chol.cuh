@@ -168,12 +168,15 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
         double x[8];
 #pragma unroll
         for (int i = 0; i < 8; ++i) x[i] = i == jc ? 1.0 : 0.0;
+        int bad = -1;                    // first pivot of this mini-block that is not positive and finite
 #pragma unroll
         for (int p = 0; p < 8; ++p) {
-            double d = m[p][p];
-            const bool ok = d > 0.0 && isfinite(d);
-            if (!ok && reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + p);
-            d = ok ? d : 1.0;
+            // A bad pivot is replaced by 1 and remembered; the report is made after the chain, so that the eight steps
+            // stay one straight line of code.
+            const double d0 = m[p][p];
+            const bool ok = d0 > 0.0 && d0 < 1.0e300;
+            bad = (!ok && bad < 0) ? p : bad;
+            const double d = ok ? d0 : 1.0;
             const double rs = rsqrt(d);
             const double inv = rs * rs;
             const double tx = x[p] * inv;
@@ -190,6 +193,7 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
 #pragma unroll
             for (int p = 0; p < 8; ++p) Wbuf[warp * 64 + p * 8 + lane] = x[p];    // W[p][j] = (U_M^-T)[p][j]
         }
+        if (bad >= 0 && reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + bad);
     }
     __syncthreads();
     const double* wb = Wbuf + (warp & 3) * 64;
