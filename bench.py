@@ -39,9 +39,9 @@ INT8_OVER_BF16 = 2.0                                   # nominal dense 4.5 / 2.2
 # profiles/, on the bench workload (Gram: scaled from the 16384-column capture by the calibration columns processed).
 # Each entry names the kernel sources it was taken with; when they have changed since, the traffic is reported as null.
 NCU_TRAFFIC = {
-    "chol_coop": {"bytes_per_launch": (42.42e6 + 4.32e6 + 21.78e6 + 0.91e6) / 2, "sources": ["chol.cuh", "dgemm.cuh"],
-                  "sha256_16": "1739f1df003b8abe"},
-    "sweep_coop": {"bytes_per_launch": 26.26e6 + 0.005e6, "sources": ["colloop.cuh"], "sha256_16": "f7a0d8df9c4618f0"},
+    "chol_coop": {"bytes_per_launch": (42.40e6 + 5.05e6 + 21.75e6 + 1.42e6) / 2, "sources": ["chol.cuh", "dgemm.cuh"],
+                  "sha256_16": "63d4585579b6af11"},
+    "sweep_coop": {"bytes_per_launch": 26.26e6 + 0.009e6, "sources": ["colloop.cuh"], "sha256_16": "f7a0d8df9c4618f0"},
     "gram_i8_tcgen05": {"bytes_per_launch": (512.6e6 + 42.8e6) * 4096 / 16384, "sources": ["gram.cuh"],
                         "sha256_16": "ad393485f71b6ece"},
 }
