@@ -24,7 +24,16 @@ inline int grid_x_for(int n, int threads) {
     return g < 1 ? 1 : (g > 1024 ? 1024 : g);
 }
 
-size_t loss_partials_count(int rows, int cols) { return (size_t)cdiv(rows, 64) * cdiv(cols, 64); }
+// The loss product is cut along k into as many slices as it takes to put about two CTAs on every SM.
+constexpr int kLossMaxSplit = 8;
+int loss_ksplit(int rows, int cols) {
+    const long ctas = (long)cdiv(rows, 64) * ((cdiv(cols, 64) + 1) / 2);
+    const long want = (2 * 148 + ctas - 1) / ctas;
+    return (int)(want < 1 ? 1 : (want > kLossMaxSplit ? kLossMaxSplit : want));
+}
+size_t loss_partials_count(int rows, int cols) {
+    return (size_t)kLossMaxSplit * cdiv(rows, 64) * cdiv(cols, 64);
+}
 
 // Built-in scratch of ptq_sensitivity_order_static: lives in every device that loads the library, until exit.
 constexpr size_t kStaticScratchDoubles = PTQ_STATIC_SCRATCH_BYTES / sizeof(double);
@@ -314,10 +323,11 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
         g.B = H_undamped; g.ldb = n; g.b_trans = 0;
         g.M = rows; g.N = n; g.K = n;
         g.D = dW; g.ldd = n; g.partials = partials;
+        g.ksplit = loss_ksplit(rows, n);
         dim3 grid;
         st = launch_dgemm(K_DGEMM_LOSS, g, 1, stream, 64, &grid);
         if (st) return st;
-        { Launch l(K_SUM_PARTIALS, stream); sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y), 0.5, loss_out); }
+        { Launch l(K_SUM_PARTIALS, stream); sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y * grid.z), 0.5, loss_out); }
     }
     return launch_status();
 }

@@ -30,6 +30,9 @@ struct GemmParams {
     const double* D;
     int64_t ldd;
     double* partials;
+    // ksplit > 1 (reduction epilogue only, one batch): blockIdx.z selects one of ksplit slices of the tile's k range;
+    // every slice writes its own partial sum, which is all a sum over k needs
+    int ksplit;
 };
 
 constexpr int kGemmBK = 16;
@@ -90,6 +93,16 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
     else if (p.kbeg_mode == 2) kbeg = i0;
     kbeg = (kbeg / BK) * BK;
     if (p.kend_mode == 1 && j0 + BT < kend) kend = j0 + BT;
+    bool double_at_end = false;
+    if (p.ksplit > 1) {
+        const int len = ((kend - kbeg + BK - 1) / BK + p.ksplit - 1) / p.ksplit * BK;
+        kbeg += z * len;
+        if (kbeg + len < kend) kend = kbeg + len;
+        // a slice that ends before the tile's own column block lies entirely in the part that counts twice
+        double_at_end = p.sym_double && kend <= j0;
+        z = 0;
+    }
+    const int zp = p.ksplit > 1 ? (int)blockIdx.z : z;          // index of the partial sum
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int wm0 = (warp >> 2) * WTM, wn0 = (warp & 3) * WTN;
@@ -169,6 +182,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
     cp_async_wait<0>();
 
     if (p.partials) {
+        const double wgt = double_at_end ? 2.0 : 1.0;
         double s = 0.0;
 #pragma unroll
         for (int a = 0; a < FM; ++a) {
@@ -190,7 +204,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
             __syncthreads();
         }
         if (tid == 0)
-            p.partials[((int64_t)z * nby + by) * nbx + bx] = red[0];
+            p.partials[((int64_t)zp * nby + by) * nbx + bx] = wgt * red[0];
         __syncthreads();
         return;
     }
@@ -255,7 +269,7 @@ inline int launch_dgemm(int kernel_id, const GemmParams& p, int batches, cudaStr
         const long tiles128 = (long)cdiv(p.M, 128) * cdiv(p.N, 128) * batches / (p.upper_only ? 2 : 1);
         bt = tiles128 >= 2 * 148 ? 128 : 64;
     }
-    dim3 grid(cdiv(p.N, bt), cdiv(p.M, bt), batches);
+    dim3 grid(cdiv(p.N, bt), cdiv(p.M, bt), p.ksplit > 1 ? p.ksplit : batches);
     if (grid_out) *grid_out = grid;          // the tile grid (what the partials are indexed by)
     if (p.sym_double) grid.x = (grid.x + 1) / 2;
     Launch scope(kernel_id, stream);
