@@ -156,6 +156,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
     double* Bb = Ea + kSweepRows * kSweepLd;                           // [2][64][68] MMA operand B: U[e, b']
     uint8_t* Cs = reinterpret_cast<uint8_t*>(Bb + 2 * kNB * kSweepLd); // [32][68] codes of the block
     int* s_flag = reinterpret_cast<int*>(Cs + kSweepRows * (kNB + 4));
+    volatile int* s_pub = s_flag + 1;                                  // last piece of E this CTA has announced
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rows = prm.rows, n = prm.n;
@@ -286,7 +287,19 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         if (cpg > 1) {
                             __threadfence();
                             __syncwarp();
-                            if (lane == 0) atomicExch(&prm.flags[g], (unsigned)(8 * b + m + 1));
+                            if (lane == 0) {
+                                // The counter must rise in order: piece m leaves only after piece m - 1 of this block
+                                // (whose fence may have taken longer than this warp's whole chain), else a reader
+                                // could be told of columns that are not visible yet, or see the counter fall back.
+                                if (m > 0) {
+                                    const long long t0 = clock64();
+                                    while (*s_pub != 8 * b + m) {
+                                        if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); break; }
+                                    }
+                                }
+                                atomicExch(&prm.flags[g], (unsigned)(8 * b + m + 1));
+                                *s_pub = 8 * b + m + 1;
+                            }
                         }
                     } else {
                         // rank-8 update of this warp's columns: blk -= d (U'[8 m .. 8 m + 7][8 warp .. 8 warp + 7])
