@@ -79,6 +79,22 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n);
 int ptq_hessian_accumulate(double *H, const float *X, int cols, int n, int64_t ldx, void *ws, size_t ws_bytes,
                            int32_t *status, void *stream);
 
+/*
+ * The same accumulation for a convolutional layer, straight from the layer's input (Sec. 3: for a convolution d_col
+ * is the number of weights of one filter, channels * kh * kw, and the columns of X are the input patches those
+ * weights see).  With out_h = (height + 2 pad - kh) / stride + 1 (out_w alike), cols = channels * kh * kw and
+ * n = batch * out_h * out_w:
+ *     X[(c * kh + ki) * kw + kj][(b * out_h + oy) * out_w + ox] = act[b][c][oy * stride + ki - pad][ox * stride + kj - pad]
+ * (zero outside the image), H += 2 X X^T.  The patches are never written out: the slicing pass reads act in place.
+ *   H    [cols x cols] float64, in/out (row and column order: channel-major, then ki, then kj, the layout of a
+ *        convolution weight [out_channels][channels][kh][kw] flattened per filter)
+ *   act  [batch][channels][height][width] float32, contiguous
+ * Workspace: ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE, 0, cols, n).  Calling it once per calibration batch
+ * accumulates over batches.  Sizes beyond cols = 2^20 or n = 2^30 return PTQ_ERR_UNSUPPORTED.
+ */
+int ptq_hessian_accumulate_conv(double *H, const float *act, int batch, int channels, int height, int width, int kh,
+                                int kw, int stride, int pad, void *ws, size_t ws_bytes, int32_t *status, void *stream);
+
 /* Same contract, computed with float64 FMAs (cross-check of the tensor-core path). */
 int ptq_hessian_accumulate_f64(double *H, const float *X, int cols, int n, int64_t ldx, void *ws, size_t ws_bytes,
                                int32_t *status, void *stream);

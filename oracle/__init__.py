@@ -55,6 +55,7 @@ def lib():
         L.oracle_num_threads.restype = c_int
         L.oracle_hessian_accumulate.argtypes = [pd, pf, c_int, c_int, c_int64]
         L.oracle_hessian_entry.argtypes = [pf, c_int, c_int64, c_int, c_int]
+        L.oracle_unfold.argtypes = [pf, pf] + [c_int] * 8
         L.oracle_hessian_entry.restype = c_double
         L.oracle_prepare_hinv.argtypes = [pd, c_int, c_int, c_double, pd, pd, pd, POINTER(c_int)]
         L.oracle_minmax_grid.argtypes = [pf, c_int, c_int, c_int64, c_int, pf, pf]
@@ -93,6 +94,25 @@ def hessian_accumulate(X, H=None):
     if st:
         raise OracleError(st, "hessian_accumulate")
     return H
+
+
+def unfold(act, kh, kw, stride=1, pad=0):
+    """Input patches of a convolution as the columns of X (Sec. 3): act [batch, channels, height, width] float32 ->
+    X [channels kh kw, batch out_h out_w] float32, rows ordered like a flattened filter (channel, ki, kj)."""
+    act = np.ascontiguousarray(act, dtype=np.float32)
+    assert act.ndim == 4
+    b, c, h, w = act.shape
+    oh, ow = (h + 2 * pad - kh) // stride + 1, (w + 2 * pad - kw) // stride + 1
+    X = np.empty((c * kh * kw, b * oh * ow), dtype=np.float32)
+    st = lib().oracle_unfold(_p(X, c_float), _p(act, c_float), b, c, h, w, int(kh), int(kw), int(stride), int(pad))
+    if st:
+        raise OracleError(st, "unfold")
+    return X
+
+
+def hessian_accumulate_conv(act, kh, kw, stride=1, pad=0, H=None):
+    """H += 2 X X^T with X = unfold(act): the Hessian of a convolutional layer (Sec. 3, Eq. 2)."""
+    return hessian_accumulate(unfold(act, kh, kw, stride, pad), H)
 
 
 def hessian_entry(X, i, j) -> float:

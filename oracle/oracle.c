@@ -45,6 +45,38 @@ int oracle_num_threads(void) {
 }
 
 /* ---------------------------------------------------------------------------------------
+ * Sec. 3: for a convolutional layer d_col is the number of weights of one filter, so the
+ * columns of X are the input patches those weights see.  Writes them out by definition:
+ *   X[(c*kh + ki)*kw + kj][(b*oh + oy)*ow + ox] = act[b][c][oy*stride + ki - pad][ox*stride + kj - pad]
+ * (zero outside the image), act = [batch][channels][height][width], X = [channels*kh*kw][batch*oh*ow],
+ * oh = (height + 2 pad - kh)/stride + 1, ow alike.  No arithmetic: the Hessian of a convolution
+ * is oracle_hessian_accumulate of this matrix.
+ * ------------------------------------------------------------------------------------- */
+int oracle_unfold(float *X, const float *act, int batch, int channels, int height, int width, int kh, int kw,
+                  int stride, int pad) {
+    if (!X || !act || batch < 1 || channels < 1 || height < 1 || width < 1 || kh < 1 || kw < 1 || stride < 1 ||
+        pad < 0 || height + 2 * pad < kh || width + 2 * pad < kw)
+        return ORACLE_ERR_INVALID_ARG;
+    const int oh = (height + 2 * pad - kh) / stride + 1, ow = (width + 2 * pad - kw) / stride + 1;
+    const size_t n = (size_t)batch * oh * ow;
+    for (int c = 0; c < channels; ++c)
+        for (int ki = 0; ki < kh; ++ki)
+            for (int kj = 0; kj < kw; ++kj) {
+                float *row = X + ((size_t)(c * kh + ki) * kw + kj) * n;
+                for (int b = 0; b < batch; ++b)
+                    for (int oy = 0; oy < oh; ++oy)
+                        for (int ox = 0; ox < ow; ++ox) {
+                            const int iy = oy * stride + ki - pad, ix = ox * stride + kj - pad;
+                            float v = 0.0f;
+                            if (iy >= 0 && iy < height && ix >= 0 && ix < width)
+                                v = act[(((size_t)b * channels + c) * height + iy) * width + ix];
+                            row[((size_t)b * oh + oy) * ow + ox] = v;
+                        }
+            }
+    return ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------------------------------
  * Sec. 3, Eq. 2: the layer error is ||W X - What X||^2, so its second derivative with
  * respect to one row of W is H = 2 X X^T.  Accumulates H += 2 * X X^T.
  * Each H[i][j] is the serial sum over n = 0..n-1 of X[i][n] * X[j][n].

@@ -186,7 +186,29 @@ int ptq_hessian_accumulate(double* H, const float* X, int cols, int n, int64_t l
     if (!H || !X || cols < 1 || n < 1 || ldx < n) return PTQ_ERR_INVALID_ARG;
     if (!aligned16(H) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE, 0, cols, n)) return PTQ_ERR_WORKSPACE;
-    return gram_accumulate(H, X, cols, n, ldx, ws, status, stream);
+    GramSource src{};
+    src.base = X; src.ldx = ldx;
+    return gram_accumulate(H, src, cols, n, ws, status, stream);
+}
+
+int ptq_hessian_accumulate_conv(double* H, const float* act, int batch, int channels, int height, int width, int kh,
+                                int kw, int stride, int pad, void* ws, size_t ws_bytes, int32_t* status,
+                                void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!H || !act || batch < 1 || channels < 1 || height < 1 || width < 1 || kh < 1 || kw < 1 || stride < 1 || pad < 0)
+        return PTQ_ERR_INVALID_ARG;
+    if (height + 2 * pad < kh || width + 2 * pad < kw) return PTQ_ERR_INVALID_ARG;
+    const int64_t oh = (height + 2 * pad - kh) / stride + 1, ow = (width + 2 * pad - kw) / stride + 1;
+    const int64_t cols64 = (int64_t)channels * kh * kw, n64 = (int64_t)batch * oh * ow;
+    if (cols64 > (1 << 20) || n64 > (int64_t)1 << 30) return PTQ_ERR_UNSUPPORTED;
+    const int cols = (int)cols64, n = (int)n64;
+    if (!aligned16(H) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE, 0, cols, n)) return PTQ_ERR_WORKSPACE;
+    GramSource src{};
+    src.base = act; src.conv = 1;
+    src.channels = channels; src.height = height; src.width = width;
+    src.kh = kh; src.kw = kw; src.stride = stride; src.pad = pad; src.oh = (int)oh; src.ow = (int)ow;
+    return gram_accumulate(H, src, cols, n, ws, status, stream);
 }
 
 int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, double* Hinv, double* Hinv_diag,

@@ -44,8 +44,42 @@ inline size_t gram_workspace_bytes(int cols, int n) {
 }
 
 // ------------------------------------------------------------------------------------------------------------
+// Where the rows of X come from.  Either a plain [cols x n] matrix, or the input of a convolution whose unfolded
+// patches ARE the columns of X (Sec. 3: for a convolutional layer d_col is the number of weights of one filter, so row
+// (c, ki, kj) of X holds, for every image b and output position (oy, ox), the input value that weight multiplies):
+//     X[(c kh + ki) kw + kj][(b OH + oy) OW + ox] = act[b][c][oy stride + ki - pad][ox stride + kj - pad]   (0 outside)
+// The patches are never materialised in float32: the slicing pre-pass reads the activations in place.
+// ------------------------------------------------------------------------------------------------------------
+struct GramSource {
+    const float* base;      // X, or the activations [batch][channels][height][width]
+    int64_t ldx;            // matrix: row stride
+    int conv;               // 0: matrix, 1: convolution input
+    int channels, height, width, kh, kw, stride, pad, oh, ow;
+    int col0;               // first calibration column of this launch
+};
+
+// ------------------------------------------------------------------------------------------------------------
 // Slicing pre-pass: one CTA per (padded) row.
 // ------------------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) gram_split_conv_kernel(GramSource src, int cols, int n, int cols_pad, int n_pad,
+                                                               int8_t* __restrict__ Q, int32_t* __restrict__ shifts,
+                                                               int32_t* status);
+
+__device__ __forceinline__ void gram_pack4(const long long (&v)[4], uint32_t (&packed)[kSlices]) {
+#pragma unroll
+    for (int s = 0; s < kSlices; ++s) packed[s] = 0u;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        long long t = v[u];
+#pragma unroll
+        for (int s = kSlices - 1; s >= 0; --s) {          // least significant digit first
+            const long long d = ((t + 128) & 255) - 128;  // balanced digit in [-128, 127]
+            t = (t - d) >> 8;
+            packed[s] |= ((uint32_t)(d & 255)) << (8 * u);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256) gram_split_kernel(const float* __restrict__ X, int cols, int n, int64_t ldx,
                                                           int cols_pad, int n_pad, int vec_ok,
                                                           int8_t* __restrict__ Q, int32_t* __restrict__ shifts,
@@ -98,18 +132,92 @@ __global__ void __launch_bounds__(256) gram_split_kernel(const float* __restrict
             v[u] = __double2ll_rn(scalbn((double)xv, sh));
         }
         uint32_t packed[kSlices];
+        gram_pack4(v, packed);
 #pragma unroll
-        for (int s = 0; s < kSlices; ++s) packed[s] = 0u;
+        for (int s = 0; s < kSlices; ++s) *reinterpret_cast<uint32_t*>(q0 + s * plane + k) = packed[s];
+    }
+}
+
+// The same pre-pass reading the input of a convolution in place (see GramSource).  Thread t walks the calibration
+// columns 4 t .. 4 t + 3, 4 t + 1024 .., keeping (image, output row, output column) up to date by carries.
+struct ConvCursor {
+    int b, oy, ox;
+    __device__ __forceinline__ void set(const GramSource& s, int col) {
+        const int per = s.oh * s.ow;
+        b = col / per;
+        const int r = col - b * per;
+        oy = r / s.ow;
+        ox = r - oy * s.ow;
+    }
+    __device__ __forceinline__ void next(const GramSource& s) {
+        if (++ox == s.ow) { ox = 0; if (++oy == s.oh) { oy = 0; ++b; } }
+    }
+};
+__device__ __forceinline__ float conv_fetch(const GramSource& s, const float* __restrict__ plane0, const ConvCursor& c,
+                                            int ki, int kj) {
+    const int iy = c.oy * s.stride + ki - s.pad, ix = c.ox * s.stride + kj - s.pad;
+    if ((unsigned)iy >= (unsigned)s.height || (unsigned)ix >= (unsigned)s.width) return 0.f;
+    return plane0[((int64_t)c.b * s.channels * s.height + iy) * s.width + ix];
+}
+
+__global__ void __launch_bounds__(256) gram_split_conv_kernel(GramSource src, int cols, int n, int cols_pad, int n_pad,
+                                                               int8_t* __restrict__ Q, int32_t* __restrict__ shifts,
+                                                               int32_t* status) {
+    __shared__ float smax[256];
+    __shared__ int sbad;
+    const int row = blockIdx.x;
+    const size_t plane = (size_t)cols_pad * n_pad;
+    int8_t* q0 = Q + (size_t)row * n_pad;
+    if (row >= cols) {   // padding rows: zeros
+        for (int k = threadIdx.x * 4; k < n_pad; k += 1024)
+#pragma unroll
+            for (int s = 0; s < kSlices; ++s) *reinterpret_cast<uint32_t*>(q0 + s * plane + k) = 0u;
+        if (threadIdx.x == 0) shifts[row] = 0;
+        return;
+    }
+    if (threadIdx.x == 0) sbad = 0;
+    __syncthreads();
+    const int kk2 = src.kh * src.kw;
+    const int ch = row / kk2, rem = row - ch * kk2;
+    const int ki = rem / src.kw, kj = rem - ki * src.kw;
+    const float* plane0 = src.base + (int64_t)ch * src.height * src.width;     // channel ch of image 0
+    float m = 0.f;
+    bool bad = false;
+    for (int k = threadIdx.x * 4; k < n; k += 1024) {
+        ConvCursor cur;
+        cur.set(src, src.col0 + k);
+        for (int u = 0; u < 4 && k + u < n; ++u) {
+            const float xv = conv_fetch(src, plane0, cur, ki, kj);
+            bad |= !isfinite(xv);
+            m = fmaxf(m, fabsf(xv));
+            cur.next(src);
+        }
+    }
+    if (bad) sbad = 1;
+    smax[threadIdx.x] = m;
+    __syncthreads();
+    for (int w = 128; w > 0; w >>= 1) {
+        if (threadIdx.x < w) smax[threadIdx.x] = fmaxf(smax[threadIdx.x], smax[threadIdx.x + w]);
+        __syncthreads();
+    }
+    const float rowmax = smax[0];
+    const bool rowbad = sbad != 0;
+    if (rowbad && threadIdx.x == 0) report(status, PTQ_ERR_NONFINITE, row);
+    int sh = 0;
+    if (rowmax > 0.f && !rowbad) sh = kShiftTarget - (ilogbf(rowmax) + 1);   // |x| 2^sh < 2^46
+    if (threadIdx.x == 0) shifts[row] = sh;
+    for (int k = threadIdx.x * 4; k < n_pad; k += 1024) {
+        long long v[4];
+        ConvCursor cur;
+        cur.set(src, src.col0 + k);
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            long long t = v[u];
-#pragma unroll
-            for (int s = kSlices - 1; s >= 0; --s) {          // least significant digit first
-                const long long d = ((t + 128) & 255) - 128;  // balanced digit in [-128, 127]
-                t = (t - d) >> 8;
-                packed[s] |= ((uint32_t)(d & 255)) << (8 * u);
-            }
+            const float xv = (k + u < n && !rowbad) ? conv_fetch(src, plane0, cur, ki, kj) : 0.f;
+            v[u] = __double2ll_rn(scalbn((double)xv, sh));
+            cur.next(src);
         }
+        uint32_t packed[kSlices];
+        gram_pack4(v, packed);
 #pragma unroll
         for (int s = 0; s < kSlices; ++s) *reinterpret_cast<uint32_t*>(q0 + s * plane + k) = packed[s];
     }
@@ -455,7 +563,7 @@ inline int make_slice_map(CUtensorMap* m, int8_t* Q, int cols_pad, int n_pad, in
     return r == CUDA_SUCCESS ? PTQ_OK : PTQ_ERR_CUDA;
 }
 
-inline int gram_accumulate(double* H, const float* X, int cols, int n, int64_t ldx, void* ws, int32_t* status,
+inline int gram_accumulate(double* H, GramSource src, int cols, int n, void* ws, int32_t* status,
                            cudaStream_t stream) {
     static bool attr_done = false;
     static int num_sms = 0;
@@ -480,11 +588,16 @@ inline int gram_accumulate(double* H, const float* X, int cols, int n, int64_t l
     for (int c0 = 0; c0 < n; c0 += kGramMaxChunk) {
         const int nc = n - c0 < kGramMaxChunk ? n - c0 : kGramMaxChunk;
         const int n_pad = cdiv(nc, 128) * 128;
-        const int vec_ok = (aligned16(X) && (ldx & 3) == 0) ? 1 : 0;
         {
             Launch l(K_GRAM_SPLIT, stream);
-            gram_split_kernel<<<cols_pad, 256, 0, stream>>>(X + c0, cols, nc, ldx, cols_pad, n_pad, vec_ok, Q, shifts,
-                                                            status);
+            if (src.conv) {
+                src.col0 = c0;
+                gram_split_conv_kernel<<<cols_pad, 256, 0, stream>>>(src, cols, nc, cols_pad, n_pad, Q, shifts, status);
+            } else {
+                const int vec_ok = (aligned16(src.base) && (src.ldx & 3) == 0) ? 1 : 0;
+                gram_split_kernel<<<cols_pad, 256, 0, stream>>>(src.base + c0, cols, nc, src.ldx, cols_pad, n_pad, vec_ok,
+                                                                Q, shifts, status);
+            }
         }
         CUtensorMap mapA, mapB;
         int st = make_slice_map(&mapA, Q, cols_pad, n_pad, kGramTM);

@@ -3,6 +3,7 @@
     python -m paper_2509_05576_b200.layer_set_run --config 3            # the 54 ResNet-50-shaped layers, 4-bit
     python -m paper_2509_05576_b200.layer_set_run --config 4 --bits 8   # the YOLOv5s-shaped stack
     python -m paper_2509_05576_b200.layer_set_run --config 5 --bits 4   # square / wide scaling shapes
+    python -m paper_2509_05576_b200.layer_set_run --config 6            # ResNet-18-shaped (7: ResNet-34-shaped)
 
 Every layer goes through the five C-ABI calls (Hessian, damped inverse, grid, scores + order, sweep); each call is
 bracketed by CUDA events on the launching stream, an L2-sized buffer is rewritten before every timed repetition.
@@ -47,7 +48,7 @@ def stage_work(spec):
 
 def main(argv=None):
     ap = argparse.ArgumentParser()
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7])
     ap.add_argument("--bits", type=int, default=None, help="bit-width filter for configs 4 and 5")
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--limit", type=int, default=0, help="only the first LIMIT layers (0: all)")

@@ -22,7 +22,7 @@ DAMP_REL_MEAN_DIAG, DAMP_ABS = 0, 1
 SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
 CALL_HESSIAN_ACCUMULATE, CALL_PREPARE_HINV, CALL_SENSITIVITY_ORDER, CALL_QUANTIZE_LAYER, CALL_HESSIAN_ACCUMULATE_F64 = range(5)
 
-EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
+EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_conv", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
            "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_sensitivity_order_static", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
            "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
 
@@ -53,6 +53,8 @@ def lib():
         L.ptq_workspace_bytes.restype = c_size_t
         for name in ("ptq_hessian_accumulate", "ptq_hessian_accumulate_f64"):
             getattr(L, name).argtypes = [vp, vp, c_int, c_int, c_int64, vp, c_size_t, vp, vp]
+        L.ptq_hessian_accumulate_conv.argtypes = [vp, vp, c_int, c_int, c_int, c_int, c_int, c_int, c_int, c_int, vp,
+                                                  c_size_t, vp, vp]
         L.ptq_prepare_hinv.argtypes = [vp, c_int, c_int, c_double, vp, vp, vp, vp, c_size_t, vp, vp]
         L.ptq_minmax_grid.argtypes = [vp, c_int, c_int, c_int64, c_int, vp, vp, vp, vp]
         L.ptq_sensitivity_order.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, c_size_t,
@@ -169,6 +171,28 @@ def hessian_accumulate(H, X, ws, status, stream=None, f64=False):
            "ptq_hessian_accumulate")
 
 
+def conv_unfolded_shape(act_shape, kh, kw, stride=1, pad=0):
+    """(cols, n) of the unfolded input of a convolution: channels kh kw rows, batch out_h out_w columns."""
+    b, c, h, w = act_shape
+    oh, ow = (h + 2 * pad - kh) // stride + 1, (w + 2 * pad - kw) // stride + 1
+    return c * kh * kw, b * oh * ow
+
+
+def hessian_accumulate_conv(H, act, kh, kw, stride, pad, ws, status, stream=None):
+    """H += 2 X X^T with X the unfolded patches of act [batch, channels, height, width] (Sec. 3), read in place."""
+    _dev(H, torch.float64, "H"); _dev(act, torch.float32, "act")
+    if act.dim() != 4 or not act.is_contiguous():
+        raise ValueError("act must be contiguous [batch, channels, height, width]")
+    b, c, h, w = act.shape
+    cols, n = conv_unfolded_shape(act.shape, kh, kw, stride, pad)
+    if H.shape != (cols, cols) or not H.is_contiguous():
+        raise ValueError("H must be contiguous [channels kh kw, channels kh kw]")
+    buf = ws.get(workspace_bytes(CALL_HESSIAN_ACCUMULATE, 0, cols, n))
+    _check(lib().ptq_hessian_accumulate_conv(_ptr(H), _ptr(act), b, c, h, w, int(kh), int(kw), int(stride), int(pad),
+                                             _ptr(buf), buf.numel(), _ptr(status), _stream(stream)),
+           "ptq_hessian_accumulate_conv")
+
+
 def prepare_hinv(H, damp, damp_mode, Hinv, Hinv_diag, lambda_out, ws, status, stream=None):
     """Hinv = (H + lambda I)^-1 (Sec. 5 item 1); also its diagonal and lambda (device scalars)."""
     _dev(H, torch.float64, "H"); _dev(Hinv, torch.float64, "Hinv")
@@ -240,10 +264,13 @@ class LayerBuffers:
 
 
 def quantize_layer_full(W, X, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG, score_mode=SCORE_QERR, bufs=None, ws=None,
-                        stream=None, want_loss=True, events=None, gram_f64=False):
+                        stream=None, want_loss=True, events=None, gram_f64=False, conv=None):
     """The whole hot path on one layer (all device-side, asynchronous on the stream):
     Hessian -> damped inverse -> grid -> scores + order -> column sweep -> codes, What, loss.
 
+    ``conv``: None for a layer given by its input matrix X [cols, n]; for a convolution ``(kh, kw, stride, pad)``,
+    and X is then the layer's input [batch, channels, height, width] or a list of such calibration batches, read in
+    place by ``ptq_hessian_accumulate_conv`` (W is the weight flattened per filter, [out_channels, channels kh kw]).
     ``events``: optional list receiving (stage name, start event, end event) for per-stage timing.
     Returns the LayerBuffers holding the outputs; call ``check_status(bufs.status)`` after synchronising.
     """
@@ -266,7 +293,13 @@ def quantize_layer_full(W, X, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG, sco
     with torch.cuda.stream(s):
         st.zero_()
         bufs.H.zero_()
-        timed("hessian", lambda: hessian_accumulate(bufs.H, X, ws, st, s, f64=gram_f64))
+        if conv is None:
+            timed("hessian", lambda: hessian_accumulate(bufs.H, X, ws, st, s, f64=gram_f64))
+        else:
+            kh, kw, stride, pad = conv
+            batches = X if isinstance(X, (list, tuple)) else [X]
+            timed("hessian", lambda: [hessian_accumulate_conv(bufs.H, a, kh, kw, stride, pad, ws, st, s)
+                                      for a in batches])
         timed("inverse", lambda: prepare_hinv(bufs.H, damp, damp_mode, bufs.Hinv, bufs.Hinv_diag, bufs.lam, ws, st, s))
         timed("grid", lambda: minmax_grid(W, bits, bufs.scale, bufs.zero, st, s))
         timed("order", lambda: sensitivity_order(W, bufs.Hinv_diag, bufs.scale, bufs.zero, bits, score_mode, bufs.S,

@@ -71,6 +71,38 @@ def test_hessian_accumulates_over_chunks():
 
 
 # ------------------------------------------------------------------ damped inverse (Sec. 5 item 1)
+@pytest.mark.parametrize("spec", wl.conv_cases(), ids=lambda s: s.name)
+def test_unfold_matches_library_unfold(spec):
+    """The patch matrix of a convolution (Sec. 3) against torch's unfold, a library routine."""
+    import torch
+    _, act = wl.make_conv_layer(spec)
+    X = oracle.unfold(act, spec.kh, spec.kw, spec.stride, spec.pad)
+    assert X.shape == (spec.cols, spec.n)
+    ref = torch.nn.functional.unfold(torch.from_numpy(act), (spec.kh, spec.kw), stride=spec.stride, padding=spec.pad)
+    ref = ref.permute(1, 0, 2).reshape(spec.cols, -1).numpy()            # [cols, batch * positions]
+    assert np.array_equal(X, ref)
+
+
+@pytest.mark.parametrize("spec", wl.conv_cases()[:4] + wl.conv_cases()[5:], ids=lambda s: s.name)
+def test_conv_hessian_is_energy_of_the_convolution_output(spec):
+    """For any filter w, 1/2 w^T H w = ||w X||^2 is the squared norm of the convolution's output map, which torch's
+    conv2d computes without ever forming patches: pins the row order (channel, ki, kj), stride and padding at once."""
+    import torch
+    W, act = wl.make_conv_layer(spec)
+    H = oracle.hessian_accumulate_conv(act, spec.kh, spec.kw, spec.stride, spec.pad)
+    assert np.array_equal(H, H.T)
+    w = W[:3].astype(np.float64)
+    out = torch.nn.functional.conv2d(torch.from_numpy(act).double(),
+                                     torch.from_numpy(w).reshape(3, spec.channels, spec.kh, spec.kw),
+                                     stride=spec.stride, padding=spec.pad).numpy()
+    for r in range(3):
+        energy = float(np.sum(out[:, r] ** 2))
+        assert abs(0.5 * w[r] @ H @ w[r] - energy) <= 1e-11 * energy
+    # two filters at once: the cross term, so that a transposed or permuted H would show
+    cross = float(np.sum(out[:, 0] * out[:, 1]))
+    assert abs(0.5 * w[0] @ H @ w[1] - cross) <= 1e-11 * np.sqrt(np.sum(out[:, 0] ** 2) * np.sum(out[:, 1] ** 2))
+
+
 @pytest.mark.parametrize("cols,n,seed", [(16, 64, 5), (96, 64, 6), (200, 300, 7)])
 def test_inverse_matches_lapack(cols, n, seed):
     _, X = _small_layer(4, cols, n, seed)
