@@ -47,7 +47,7 @@ inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 // separate, untimed passes.
 // ---------------------------------------------------------------------------------------------------------
 enum KernelId {
-    K_GRAM_SPLIT = 0, K_GRAM_I8, K_CONVERT_F64, K_DGEMM_GRAM, K_LAMBDA, K_DAMP_COPY, K_CHOL_COOP,
+    K_GRAM_SPLIT = 0, K_GRAM_I8, K_GRAM_FINISH, K_CONVERT_F64, K_DGEMM_GRAM, K_LAMBDA, K_DAMP_COPY, K_CHOL_COOP,
     K_DGEMM_LAUUM, K_EXTRACT_DIAG, K_MINMAX_GRID, K_SCORE_PARTIAL,
     K_SCORE_FINAL, K_RANK_SORT, K_PERM_CHECK, K_GATHER_SYM, K_GATHER_W, K_SWEEP_COOP, K_FINALIZE,
     K_DGEMM_LOSS, K_SUM_PARTIALS, K_COUNT
@@ -55,7 +55,7 @@ enum KernelId {
 
 inline const char* kernel_name(int id) {
     static const char* names[K_COUNT] = {
-        "gram_split", "gram_i8_tcgen05", "convert_f64", "dgemm_gram_f64", "lambda", "damp_copy", "chol_coop",
+        "gram_split", "gram_i8_tcgen05", "gram_finish", "convert_f64", "dgemm_gram_f64", "lambda", "damp_copy", "chol_coop",
         "dgemm_lauum", "extract_diag",
         "minmax_grid", "score_partial", "score_final", "rank_sort", "perm_check", "gather_sym", "gather_w",
         "sweep_coop", "finalize", "dgemm_loss", "sum_partials"};

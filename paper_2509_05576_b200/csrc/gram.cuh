@@ -36,11 +36,16 @@ constexpr int kGramThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM, w
 constexpr int kGramMaxChunk = 16384;       // calibration columns per launch: 6 * 2^14 * 16384 < 2^31
 constexpr int kShiftTarget = 46;
 
+constexpr int kGramSplitMaxCols = 1024;    // up to this many (padded) columns the K range may be cut across CTAs
+constexpr int kGramMaxSplit = 16;
+
 inline size_t gram_workspace_bytes(int cols, int n) {
     const size_t cols_pad = (size_t)cdiv(cols, 128) * 128;
     const int chunk = n < kGramMaxChunk ? n : kGramMaxChunk;
     const size_t n_pad = (size_t)cdiv(chunk, 128) * 128;
-    return align_up(kSlices * cols_pad * n_pad) + align_up(cols_pad * sizeof(int32_t));
+    size_t total = align_up(kSlices * cols_pad * n_pad) + align_up(cols_pad * sizeof(int32_t));
+    if (cols_pad <= (size_t)kGramSplitMaxCols) total += align_up(2 * cols_pad * cols_pad * sizeof(long long));
+    return total;
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -337,7 +342,8 @@ __device__ __forceinline__ void gram_tile_coords(int tile, int nbj, int& bi, int
 __global__ void __launch_bounds__(kGramThreads, 1)
 gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                double* __restrict__ H, int cols, int n_pad,
-               const int32_t* __restrict__ shifts, int num_tiles, int nbj, int32_t* status) {
+               const int32_t* __restrict__ shifts, int num_tiles, int nbj, int32_t* status, int ksplit,
+               unsigned long long* __restrict__ iacc, int cols_pad) {
     extern __shared__ unsigned char gram_smem_raw[];
     const uint32_t raw = smem_u32(gram_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -354,6 +360,9 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = n_pad / kGramKB;
+    // work items: (tile, slice of the K range); ksplit == 1 is the plain case
+    const int klen = (nkb + ksplit - 1) / ksplit;
+    const int num_items = num_tiles * ksplit;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kGramStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -383,10 +392,11 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 #pragma unroll
             for (int s = 0; s < kGramStages; ++s) armed[s] = -1;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
                 int bi, bj;
-                gram_tile_coords(tile, nbj, bi, bj);
-                for (int kb = 0; kb < nkb && ok; ++kb) {
+                gram_tile_coords(item / ksplit, nbj, bi, bj);
+                const int kb0 = (item % ksplit) * klen, kb1 = kb0 + klen < nkb ? kb0 + klen : nkb;
+                for (int kb = kb0; kb < kb1 && ok; ++kb) {
                     ok = mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag);
                     if (!ok) break;
                     const uint32_t sbase = base + stage * kGramStageBytes;
@@ -416,18 +426,19 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             int stage = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+            for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
                 ok = mbar_wait_bounded(acc_empty, acc_phase ^ 1u, abort_flag);   // epilogue has drained TMEM
                 if (!ok) break;
                 tc_fence_after();
-                for (int kb = 0; kb < nkb && ok; ++kb) {
+                const int kb0 = (item % ksplit) * klen, kb1 = kb0 + klen < nkb ? kb0 + klen : nkb;
+                for (int kb = kb0; kb < kb1 && ok; ++kb) {
                     ok = mbar_wait_bounded(full_bar(stage), phase, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     // Descriptors: A and B tiles share the high word; the low word is the stage's address field plus a
                     // compile-time offset per slice and per 32-byte K step, so each MMA costs two integer adds.
                     const uint32_t sb = kDescLo + ((base + stage * kGramStageBytes) >> 4);
-                    const uint32_t first = kb > 0 ? 1u : 0u;      // the first product of a group overwrites on kb == 0
+                    const uint32_t first = kb > kb0 ? 1u : 0u;    // the first product of a group overwrites
 #pragma unroll
                     for (int t = 0; t < kGroups; ++t) {
 #pragma unroll
@@ -456,9 +467,9 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         const int r_in_tile = quarter * 32 + lane;
         uint32_t acc_phase = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
             int bi, bj;
-            gram_tile_coords(tile, nbj, bi, bj);
+            gram_tile_coords(item / ksplit, nbj, bi, bj);
             ok = mbar_wait_bounded(acc_full, acc_phase, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -491,6 +502,17 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_ld16(taddr + 0 * kGramTN, r); tc_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 16; ++c) hi[c] += (long long)(int)r[c] << 16;
+                if (ksplit > 1) {
+                    // a slice of the K range: the exact integer sums go to the workspace (integer atomics commute, so
+                    // the total does not depend on the order of the slices); stored transposed, rows contiguous
+                    const size_t plane = (size_t)cols_pad * cols_pad;
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const size_t idx = (size_t)(bj * kGramTN + ch * 16 + c) * cols_pad + row;
+                        atomicAdd(iacc + idx, (unsigned long long)hi[c]);
+                        atomicAdd(iacc + plane + idx, (unsigned long long)lo[c]);
+                    }
+                }
 #pragma unroll
                 for (int c = 0; c < 16; ++c) v[ch * 16 + c] = fma((double)hi[c], 16777216.0, (double)lo[c]);
             }
@@ -499,7 +521,7 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             acc_phase ^= 1u;
             // 2. H += v 2^(41 - sh_i - sh_j).  Tiles away from the diagonal also own the mirrored entries (j, i); since H
             //    is symmetric the old value is read there, where consecutive lanes (rows i) are contiguous.
-            if (row < cols) {
+            if (row < cols && ksplit == 1) {
                 const bool straddle = (bj * kGramTN < bi * kGramTM + kGramTM);
                 const double fi = __longlong_as_double((long long)(1023 + 20 - sh_i) << 52);     // 2^(20 - sh_i)
 #pragma unroll
@@ -529,6 +551,25 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
     if (threadIdx.x == 0 && *abort_flag) report(status, PTQ_ERR_TIMEOUT, blockIdx.x);
+}
+
+// After a launch with K slices: H[i][j] += (hi 2^24 + lo) 2^(41 - sh_i - sh_j) from the integer sums, rounded once like
+// the unsliced epilogue (so the result is the same bit for bit), both triangles.
+__global__ void __launch_bounds__(256) gram_finish_kernel(const unsigned long long* __restrict__ iacc,
+                                                           double* __restrict__ H, int cols, int cols_pad,
+                                                           const int32_t* __restrict__ shifts) {
+    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (idx >= (int64_t)cols * cols) return;
+    const int col = (int)(idx / cols), row = (int)(idx - (int64_t)col * cols);       // rows run fastest
+    if (col < row) return;
+    const size_t plane = (size_t)cols_pad * cols_pad, at = (size_t)col * cols_pad + row;
+    const long long hi = (long long)iacc[at], lo = (long long)iacc[plane + at];
+    const double v = fma((double)hi, 16777216.0, (double)lo);
+    const double fi = __longlong_as_double((long long)(1023 + 20 - shifts[row]) << 52);
+    const double fj = __longlong_as_double((long long)(1023 + 21 - shifts[col]) << 52);
+    const double out = H[(int64_t)col * cols + row] + (v * fi) * fj;
+    H[(int64_t)col * cols + row] = out;
+    H[(int64_t)row * cols + col] = out;
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -582,6 +623,8 @@ inline int gram_accumulate(double* H, GramSource src, int cols, int n, void* ws,
     Carver cv(ws);
     int8_t* Q = cv.take<int8_t>(kSlices * (size_t)cols_pad * n_pad_max);
     int32_t* shifts = cv.take<int32_t>(cols_pad);
+    unsigned long long* iacc =
+        cols_pad <= kGramSplitMaxCols ? cv.take<unsigned long long>(2 * (size_t)cols_pad * cols_pad) : nullptr;
     const int nbi = cdiv(cols, kGramTM), nbj = cdiv(cols, kGramTN);
     int num_tiles = 0;
     for (int b = 0; b < nbi; ++b) num_tiles += (nbj - 2 * b) > 0 ? (nbj - 2 * b) : 0;
@@ -604,11 +647,29 @@ inline int gram_accumulate(double* H, GramSource src, int cols, int n, void* ws,
         if (st) return st;
         st = make_slice_map(&mapB, Q, cols_pad, n_pad, kGramTN);
         if (st) return st;
-        const int grid = num_tiles < num_sms ? num_tiles : num_sms;
+        // Few tiles (narrow layers): cut the K range so that every SM gets a work item.
+        int ksplit = 1;
+        const int nkb = n_pad / kGramKB;
+        if (iacc != nullptr && 2 * num_tiles <= num_sms) {
+            ksplit = num_sms / num_tiles;
+            if (ksplit > kGramMaxSplit) ksplit = kGramMaxSplit;
+            if (ksplit > nkb / 2) ksplit = nkb / 2 > 0 ? nkb / 2 : 1;
+            ksplit = cdiv(nkb, cdiv(nkb, ksplit));          // no empty slice
+        }
+        if (ksplit > 1 &&
+            cudaMemsetAsync(iacc, 0, 2 * (size_t)cols_pad * cols_pad * sizeof(unsigned long long), stream) != cudaSuccess)
+            return PTQ_ERR_CUDA;
+        const int items = num_tiles * ksplit;
+        const int grid = items < num_sms ? items : num_sms;
         {
             Launch l(K_GRAM_I8, stream);
             gram_i8_kernel<<<grid, kGramThreads, kGramSmemBytes, stream>>>(mapA, mapB, H, cols, n_pad, shifts,
-                                                                         num_tiles, nbj, status);
+                                                                         num_tiles, nbj, status, ksplit, iacc, cols_pad);
+        }
+        if (ksplit > 1) {
+            Launch l(K_GRAM_FINISH, stream);
+            gram_finish_kernel<<<(unsigned)(((int64_t)cols * cols + 255) / 256), 256, 0, stream>>>(iacc, H, cols, cols_pad,
+                                                                                              shifts);
         }
         if (cudaGetLastError() != cudaSuccess) return PTQ_ERR_CUDA;
     }
