@@ -474,18 +474,17 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         const int lgP = 6 - lgH;
         const int TP = T << lgP;
         struct Piece { double* C; const double* Bsrc; int i0, j0, tri; };
+        // pieces are asked for in ascending order, so the row of the triangular list is found by walking on from the
+        // row of the previous piece
+        int cur_r = 0, cur_start = 0;                       // row cur_r of the A list starts at tile cur_start
         auto piece_of = [&](int tp) {
             Piece pc;
             const int t = tp >> lgP;
             const int h0 = (tp & ((1 << lgP) - 1)) << lgH;
             if (t < TA) {
-                // largest r with r m - r (r - 1) / 2 <= t
-                const float mm = (float)m + 0.5f;
-                int r = (int)(mm - sqrtf(fmaxf(mm * mm - 2.0f * (float)t, 0.0f)));
-                r = r < 0 ? 0 : (r > m - 1 ? m - 1 : r);
-                while (r > 0 && r * m - r * (r - 1) / 2 > t) --r;
-                while (r + 1 < m && (r + 1) * m - (r + 1) * r / 2 <= t) ++r;
-                const int bi = row_base + r, bj = bi + (t - (r * m - r * (r - 1) / 2));
+                while (t >= cur_start + (m - cur_r)) { cur_start += m - cur_r; ++cur_r; }
+                const int r = cur_r;
+                const int bi = row_base + r, bj = bi + (t - cur_start);
                 pc.C = A; pc.Bsrc = A; pc.i0 = bi * kNB + h0; pc.j0 = bj * kNB;
                 pc.tri = bi == bj ? h0 : -1;
             } else {
