@@ -50,6 +50,10 @@ __device__ __forceinline__ void cp_async8(void* smem_dst, const void* gsrc, bool
     const int sz = valid ? 8 : 0;    // src-size 0: the 8 bytes are filled with zeros
     asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(d), "l"(gsrc), "r"(sz) : "memory");
 }
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
@@ -115,9 +119,26 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
 #pragma unroll
         for (int b = 0; b < FN; ++b) acc[a][b][0] = acc[a][b][1] = 0.0;
 
+    // operand tiles that lie inside their matrices are fetched two doubles at a time when the addresses allow it
+    const bool a_vec = (reinterpret_cast<uintptr_t>(A) & 15u) == 0 && (p.lda & 1) == 0 && i0 + BT <= M;
+    const bool b_vec = (reinterpret_cast<uintptr_t>(B) & 15u) == 0 && (p.ldb & 1) == 0 && j0 + BT <= N;
     auto load_stage = [&](int stage, int k0) {
         double* as = smem + (size_t)stage * 2 * TILE;
         double* bs = as + TILE;
+        const bool kfull = k0 + BK <= kend;
+        if (a_vec && kfull) {
+#pragma unroll
+            for (int r = 0; r < EPT / 2; ++r) {
+                const int idx = tid + r * kGemmThreads;          // pair index
+                if (a_trans == 0) {
+                    const int k = (idx & 7) * 2, m = idx >> 3;
+                    cp_async16(as + m * kGemmLdk + k, A + (int64_t)(i0 + m) * p.lda + k0 + k);
+                } else {
+                    const int m = (idx % (BT / 2)) * 2, k = idx / (BT / 2);
+                    cp_async16(as + k * LDM + m, A + (int64_t)(k0 + k) * p.lda + i0 + m);
+                }
+            }
+        } else {
 #pragma unroll
         for (int r = 0; r < EPT; ++r) {
             const int idx = tid + r * kGemmThreads;
@@ -128,6 +149,21 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
             const bool ok = gi < M && gk < kend;
             const double* src = ok ? (a_trans == 0 ? A + (int64_t)gi * p.lda + gk : A + (int64_t)gk * p.lda + gi) : A;
             cp_async8(as + off, src, ok);
+        }
+        }
+        if (b_vec && kfull) {
+#pragma unroll
+            for (int r = 0; r < EPT / 2; ++r) {
+                const int idx = tid + r * kGemmThreads;
+                if (b_trans == 1) {
+                    const int k = (idx & 7) * 2, nn = idx >> 3;
+                    cp_async16(bs + nn * kGemmLdk + k, B + (int64_t)(j0 + nn) * p.ldb + k0 + k);
+                } else {
+                    const int nn = (idx % (BT / 2)) * 2, k = idx / (BT / 2);
+                    cp_async16(bs + k * LDM + nn, B + (int64_t)(k0 + k) * p.ldb + j0 + nn);
+                }
+            }
+            return;
         }
 #pragma unroll
         for (int r = 0; r < EPT; ++r) {
