@@ -35,7 +35,7 @@ struct GemmParams {
     int ksplit;
 };
 
-constexpr int kGemmBK = 16;
+constexpr int kGemmBK = 32;
 constexpr int kGemmStages = 3;
 constexpr int kGemmThreads = 256;
 constexpr int kGemmLdk = kGemmBK + 4;   // row stride of a k-contiguous operand tile (20 = 4 mod 16: conflict-free)
@@ -131,7 +131,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
             for (int r = 0; r < EPT / 2; ++r) {
                 const int idx = tid + r * kGemmThreads;          // pair index
                 if (a_trans == 0) {
-                    const int k = (idx & 7) * 2, m = idx >> 3;
+                    const int k = (idx % (BK / 2)) * 2, m = idx / (BK / 2);
                     cp_async16(as + m * kGemmLdk + k, A + (int64_t)(i0 + m) * p.lda + k0 + k);
                 } else {
                     const int m = (idx % (BT / 2)) * 2, k = idx / (BT / 2);
@@ -143,7 +143,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
         for (int r = 0; r < EPT; ++r) {
             const int idx = tid + r * kGemmThreads;
             int m, k, off;
-            if (a_trans == 0) { k = idx & 15; m = idx >> 4; off = m * kGemmLdk + k; }
+            if (a_trans == 0) { k = idx % BK; m = idx / BK; off = m * kGemmLdk + k; }
             else { m = idx % BT; k = idx / BT; off = k * LDM + m; }
             const int gi = i0 + m, gk = k0 + k;
             const bool ok = gi < M && gk < kend;
@@ -156,7 +156,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
             for (int r = 0; r < EPT / 2; ++r) {
                 const int idx = tid + r * kGemmThreads;
                 if (b_trans == 1) {
-                    const int k = (idx & 7) * 2, nn = idx >> 3;
+                    const int k = (idx % (BK / 2)) * 2, nn = idx / (BK / 2);
                     cp_async16(bs + nn * kGemmLdk + k, B + (int64_t)(j0 + nn) * p.ldb + k0 + k);
                 } else {
                     const int nn = (idx % (BT / 2)) * 2, k = idx / (BT / 2);
@@ -169,7 +169,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
         for (int r = 0; r < EPT; ++r) {
             const int idx = tid + r * kGemmThreads;
             int n, k, off;
-            if (b_trans == 1) { k = idx & 15; n = idx >> 4; off = n * kGemmLdk + k; }
+            if (b_trans == 1) { k = idx % BK; n = idx / BK; off = n * kGemmLdk + k; }
             else { n = idx % BT; k = idx / BT; off = k * LDM + n; }
             const int gj = j0 + n, gk = k0 + k;
             const bool ok = gj < N && gk < kend;
@@ -267,7 +267,7 @@ __device__ __forceinline__ void dgemm_tile(const GemmParams& p, int bx, int by, 
 // With sym_double the grid has half as many column tiles: CTA x handles column tiles x and nbx - 1 - x, whose k ranges
 // (64 (x + 1) and 64 (nbx - x)) add up to the same length for every CTA.
 template <int BT>
-__global__ void __launch_bounds__(kGemmThreads) dgemm_kernel(GemmParams p) {
+__global__ void __launch_bounds__(kGemmThreads, BT == 64 ? 2 : 1) dgemm_kernel(GemmParams p) {
     if (p.sym_double) {
         const int nbx = (p.N + BT - 1) / BT;
         const int bx = blockIdx.x, bx2 = nbx - 1 - bx;
