@@ -35,15 +35,25 @@ constexpr int kGramThreads = 192;          // warp 0: TMA, warp 1: MMA + TMEM, w
 constexpr int kGramMaxChunk = 16384;       // calibration columns per launch: 6 * 2^14 * 16384 < 2^31
 constexpr int kShiftTarget = 46;
 
-constexpr int kGramSplitMaxCols = 1024;    // up to this many (padded) columns the K range may be cut across CTAs
-constexpr int kGramMaxSplit = 16;
+constexpr int kGramMaxSplit = 16;          // slices of the K range per tile
+constexpr int kGramMaxSplitTiles = 128;    // tiles of one launch whose K range may be cut across CTAs
+constexpr size_t kGramTileAccWords = 2 * (size_t)kGramTM * kGramTN;   // int64 words per such tile (high and low sums)
+
+inline int gram_num_tiles(int cols) {
+    const int nbi = cdiv(cols, kGramTM), nbj = cdiv(cols, kGramTN);
+    int t = 0;
+    for (int b = 0; b < nbi; ++b) t += (nbj - 2 * b) > 0 ? (nbj - 2 * b) : 0;
+    return t;
+}
 
 inline size_t gram_workspace_bytes(int cols, int n) {
     const size_t cols_pad = (size_t)cdiv(cols, 128) * 128;
     const int chunk = n < kGramMaxChunk ? n : kGramMaxChunk;
     const size_t n_pad = (size_t)cdiv(chunk, 128) * 128;
     size_t total = align_up(kSlices * cols_pad * n_pad) + align_up(cols_pad * sizeof(int32_t));
-    if (cols_pad <= (size_t)kGramSplitMaxCols) total += align_up(2 * cols_pad * cols_pad * sizeof(long long));
+    const int tiles = gram_num_tiles(cols);
+    total += align_up((size_t)(tiles < kGramMaxSplitTiles ? tiles : kGramMaxSplitTiles) * kGramTileAccWords *
+                      sizeof(long long));
     return total;
 }
 
@@ -319,8 +329,8 @@ __device__ __forceinline__ void gram_tile_coords(int tile, int nbj, int& bi, int
 __global__ void __launch_bounds__(kGramThreads, 1)
 gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB,
                double* __restrict__ H, int cols, int n_pad,
-               const int32_t* __restrict__ shifts, int num_tiles, int nbj, int32_t* status, int ksplit,
-               unsigned long long* __restrict__ iacc, int cols_pad) {
+               const int32_t* __restrict__ shifts, int num_tiles, int nbj, int32_t* status, int n_full, int ksplit,
+               unsigned long long* __restrict__ iacc) {
     extern __shared__ unsigned char gram_smem_raw[];
     const uint32_t raw = smem_u32(gram_smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u;
@@ -337,9 +347,17 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int nkb = n_pad / kGramKB;
-    // work items: (tile, slice of the K range); ksplit == 1 is the plain case
+    // Work items: the first n_full tiles whole, then the remaining tiles cut into ksplit slices of the K range each
+    // (a last, partly filled wave of tiles, or all tiles of a narrow matrix, spread over every SM this way).
     const int klen = (nkb + ksplit - 1) / ksplit;
-    const int num_items = num_tiles * ksplit;
+    const int num_items = n_full + (num_tiles - n_full) * ksplit;
+    auto item_tile = [&](int item) { return item < n_full ? item : n_full + (item - n_full) / ksplit; };
+    auto item_kb0 = [&](int item) { return item < n_full ? 0 : ((item - n_full) % ksplit) * klen; };
+    auto item_kb1 = [&](int item) {
+        if (item < n_full) return nkb;
+        const int e = item_kb0(item) + klen;
+        return e < nkb ? e : nkb;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kGramStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -371,8 +389,8 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             bool ok = true;
             for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
                 int bi, bj;
-                gram_tile_coords(item / ksplit, nbj, bi, bj);
-                const int kb0 = (item % ksplit) * klen, kb1 = kb0 + klen < nkb ? kb0 + klen : nkb;
+                gram_tile_coords(item_tile(item), nbj, bi, bj);
+                const int kb0 = item_kb0(item), kb1 = item_kb1(item);
                 for (int kb = kb0; kb < kb1 && ok; ++kb) {
                     ok = mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag);
                     if (!ok) break;
@@ -407,7 +425,7 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 ok = mbar_wait_bounded(acc_empty, acc_phase ^ 1u, abort_flag);   // epilogue has drained TMEM
                 if (!ok) break;
                 tc_fence_after();
-                const int kb0 = (item % ksplit) * klen, kb1 = kb0 + klen < nkb ? kb0 + klen : nkb;
+                const int kb0 = item_kb0(item), kb1 = item_kb1(item);
                 for (int kb = kb0; kb < kb1 && ok; ++kb) {
                     ok = mbar_wait_bounded(full_bar(stage), phase, abort_flag);
                     if (!ok) break;
@@ -446,7 +464,9 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
         bool ok = true;
         for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
             int bi, bj;
-            gram_tile_coords(item / ksplit, nbj, bi, bj);
+            const int tile = item_tile(item);
+            const bool sliced = item >= n_full && ksplit > 1;
+            gram_tile_coords(tile, nbj, bi, bj);
             ok = mbar_wait_bounded(acc_full, acc_phase, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -479,15 +499,15 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
                 tc_ld16(taddr + 0 * kGramTN, r); tc_wait_ld();
 #pragma unroll
                 for (int c = 0; c < 16; ++c) hi[c] += (long long)(int)r[c] << 16;
-                if (ksplit > 1) {
-                    // a slice of the K range: the exact integer sums go to the workspace (integer atomics commute, so
-                    // the total does not depend on the order of the slices); stored transposed, rows contiguous
-                    const size_t plane = (size_t)cols_pad * cols_pad;
+                if (sliced) {
+                    // a slice of the K range: the exact integer sums go to the tile's workspace (integer atomics commute,
+                    // so the total does not depend on the order of the slices); column-major, rows contiguous
+                    unsigned long long* acc = iacc + (size_t)(tile - n_full) * kGramTileAccWords;
 #pragma unroll
                     for (int c = 0; c < 16; ++c) {
-                        const size_t idx = (size_t)(bj * kGramTN + ch * 16 + c) * cols_pad + row;
-                        atomicAdd(iacc + idx, (unsigned long long)hi[c]);
-                        atomicAdd(iacc + plane + idx, (unsigned long long)lo[c]);
+                        const int idx = (ch * 16 + c) * kGramTM + r_in_tile;
+                        atomicAdd(acc + idx, (unsigned long long)hi[c]);
+                        atomicAdd(acc + kGramTM * kGramTN + idx, (unsigned long long)lo[c]);
                     }
                 }
 #pragma unroll
@@ -498,7 +518,7 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
             acc_phase ^= 1u;
             // 2. H += v 2^(41 - sh_i - sh_j).  Tiles away from the diagonal also own the mirrored entries (j, i); since H
             //    is symmetric the old value is read there, where consecutive lanes (rows i) are contiguous.
-            if (row < cols && ksplit == 1) {
+            if (row < cols && !sliced) {
                 const bool straddle = (bj * kGramTN < bi * kGramTM + kGramTM);
                 const double fi = __longlong_as_double((long long)(1023 + 20 - sh_i) << 52);     // 2^(20 - sh_i)
 #pragma unroll
@@ -530,23 +550,37 @@ gram_i8_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant_
     if (threadIdx.x == 0 && *abort_flag) report(status, PTQ_ERR_TIMEOUT, blockIdx.x);
 }
 
-// After a launch with K slices: H[i][j] += (hi 2^24 + lo) 2^(41 - sh_i - sh_j) from the integer sums, rounded once like
-// the unsliced epilogue (so the result is the same bit for bit), both triangles.
-__global__ void __launch_bounds__(256) gram_finish_kernel(const unsigned long long* __restrict__ iacc,
-                                                           double* __restrict__ H, int cols, int cols_pad,
-                                                           const int32_t* __restrict__ shifts) {
-    const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (idx >= (int64_t)cols * cols) return;
-    const int col = (int)(idx / cols), row = (int)(idx - (int64_t)col * cols);       // rows run fastest
-    if (col < row) return;
-    const size_t plane = (size_t)cols_pad * cols_pad, at = (size_t)col * cols_pad + row;
-    const long long hi = (long long)iacc[at], lo = (long long)iacc[plane + at];
-    const double v = fma((double)hi, 16777216.0, (double)lo);
+// After a launch with sliced tiles: for each of them, H += (hi 2^24 + lo) 2^(41 - sh_i - sh_j) from the integer sums,
+// rounded once and written exactly as the unsliced epilogue does (so the result is the same bit for bit).
+// One CTA per sliced tile and group of 16 columns, one thread per row of the tile.
+__global__ void __launch_bounds__(kGramTM) gram_finish_kernel(const unsigned long long* __restrict__ iacc,
+                                                               double* __restrict__ H, int cols, int n_full, int nbj,
+                                                               const int32_t* __restrict__ shifts) {
+    const int tile = n_full + blockIdx.x;
+    int bi, bj;
+    gram_tile_coords(tile, nbj, bi, bj);
+    const int row = bi * kGramTM + threadIdx.x;
+    if (row >= cols) return;
+    const unsigned long long* acc = iacc + (size_t)blockIdx.x * kGramTileAccWords;
+    const bool straddle = (bj * kGramTN < bi * kGramTM + kGramTM);
     const double fi = __longlong_as_double((long long)(1023 + 20 - shifts[row]) << 52);
-    const double fj = __longlong_as_double((long long)(1023 + 21 - shifts[col]) << 52);
-    const double out = H[(int64_t)col * cols + row] + (v * fi) * fj;
-    H[(int64_t)col * cols + row] = out;
-    H[(int64_t)row * cols + col] = out;
+#pragma unroll 4
+    for (int cc = 0; cc < 16; ++cc) {
+        const int c = blockIdx.y * 16 + cc, col = bj * kGramTN + c;
+        if (col >= cols) continue;
+        const long long hi = (long long)acc[c * kGramTM + threadIdx.x];
+        const long long lo = (long long)acc[kGramTM * kGramTN + c * kGramTM + threadIdx.x];
+        const double v = fma((double)hi, 16777216.0, (double)lo);
+        const double fj = __longlong_as_double((long long)(1023 + 21 - shifts[col]) << 52);
+        const double add = (v * fi) * fj;
+        if (straddle) {
+            H[(int64_t)row * cols + col] += add;
+        } else {
+            const double out = H[(int64_t)col * cols + row] + add;
+            H[(int64_t)col * cols + row] = out;
+            H[(int64_t)row * cols + col] = out;
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------------------------
@@ -584,11 +618,10 @@ inline int gram_accumulate(double* H, GramSource src, int cols, int n, void* ws,
     Carver cv(ws);
     int8_t* Q = cv.take<int8_t>(kSlices * (size_t)cols_pad * n_pad_max);
     int32_t* shifts = cv.take<int32_t>(cols_pad);
-    unsigned long long* iacc =
-        cols_pad <= kGramSplitMaxCols ? cv.take<unsigned long long>(2 * (size_t)cols_pad * cols_pad) : nullptr;
-    const int nbi = cdiv(cols, kGramTM), nbj = cdiv(cols, kGramTN);
-    int num_tiles = 0;
-    for (int b = 0; b < nbi; ++b) num_tiles += (nbj - 2 * b) > 0 ? (nbj - 2 * b) : 0;
+    const int nbj = cdiv(cols, kGramTN);
+    const int num_tiles = gram_num_tiles(cols);
+    unsigned long long* iacc = cv.take<unsigned long long>(
+        (size_t)(num_tiles < kGramMaxSplitTiles ? num_tiles : kGramMaxSplitTiles) * kGramTileAccWords);
     for (int c0 = 0; c0 < n; c0 += kGramMaxChunk) {
         const int nc = n - c0 < kGramMaxChunk ? n - c0 : kGramMaxChunk;
         const int n_pad = cdiv(nc, 128) * 128;
@@ -608,29 +641,32 @@ inline int gram_accumulate(double* H, GramSource src, int cols, int n, void* ws,
         if (st) return st;
         st = make_slice_map(&mapB, Q, cols_pad, n_pad, kGramTN);
         if (st) return st;
-        // Few tiles (narrow layers): cut the K range so that every SM gets a work item.
-        int ksplit = 1;
+        // The tiles of the last, partly filled wave (all tiles of a narrow matrix) are cut along K so that every SM
+        // gets a work item of about the same length.
         const int nkb = n_pad / kGramKB;
-        if (iacc != nullptr && 2 * num_tiles <= num_sms) {
-            ksplit = num_sms / num_tiles;
+        const int rem = num_tiles % num_sms;
+        int n_full = num_tiles, ksplit = 1;
+        if (rem > 0 && rem <= kGramMaxSplitTiles && 2 * rem <= num_sms) {
+            ksplit = num_sms / rem;
             if (ksplit > kGramMaxSplit) ksplit = kGramMaxSplit;
             if (ksplit > nkb / 2) ksplit = nkb / 2 > 0 ? nkb / 2 : 1;
             ksplit = cdiv(nkb, cdiv(nkb, ksplit));          // no empty slice
+            if (ksplit > 1) n_full = num_tiles - rem;
         }
-        if (ksplit > 1 &&
-            cudaMemsetAsync(iacc, 0, 2 * (size_t)cols_pad * cols_pad * sizeof(unsigned long long), stream) != cudaSuccess)
+        const int sliced = num_tiles - n_full;
+        if (sliced > 0 &&
+            cudaMemsetAsync(iacc, 0, (size_t)sliced * kGramTileAccWords * sizeof(unsigned long long), stream) != cudaSuccess)
             return PTQ_ERR_CUDA;
-        const int items = num_tiles * ksplit;
+        const int items = n_full + sliced * ksplit;
         const int grid = items < num_sms ? items : num_sms;
         {
             Launch l(K_GRAM_I8, stream);
             gram_i8_kernel<<<grid, kGramThreads, kGramSmemBytes, stream>>>(mapA, mapB, H, cols, n_pad, shifts,
-                                                                         num_tiles, nbj, status, ksplit, iacc, cols_pad);
+                                                                         num_tiles, nbj, status, n_full, ksplit, iacc);
         }
-        if (ksplit > 1) {
+        if (sliced > 0) {
             Launch l(K_GRAM_FINISH, stream);
-            gram_finish_kernel<<<(unsigned)(((int64_t)cols * cols + 255) / 256), 256, 0, stream>>>(iacc, H, cols, cols_pad,
-                                                                                              shifts);
+            gram_finish_kernel<<<dim3(sliced, kGramTN / 16), kGramTM, 0, stream>>>(iacc, H, cols, n_full, nbj, shifts);
         }
         if (cudaGetLastError() != cudaSuccess) return PTQ_ERR_CUDA;
     }
