@@ -193,7 +193,7 @@ def algorithmic_work(spec):
         "chol_coop": ("alu", 2 * (c ** 3 / 3.0)),                   # two Cholesky factorisations, c^3/3 flops each
         "dgemm_trtri": ("alu", c ** 3 / 3.0),
         "dgemm_lauum": ("alu", c ** 3 / 3.0),
-        "dgemm_loss": ("alu", 2.0 * r * c * c),
+        "dgemm_loss": ("alu", 1.0 * r * c * c),                     # H symmetric: half of the 2 r c^2 of the plain product
         # sweep: float64 W in and E out, codes out, the upper factor U once per 32-row group is NOT counted (L2)
         "sweep_coop": ("hbm", 8.0 * r * c + 8.0 * r * c + 1.0 * r * c + 8.0 * c * c / 2),
         "score_partial": ("hbm", 4.0 * r * c),
