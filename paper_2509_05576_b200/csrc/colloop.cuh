@@ -108,6 +108,12 @@ __device__ __forceinline__ void sweep_load_tile(double* dst, int dst_ld, const d
     }
 }
 
+__device__ __forceinline__ double ld_relaxed_f64(const double* p) {
+    double v;
+    asm volatile("ld.relaxed.gpu.global.f64 %0, [%1];" : "=d"(v) : "l"(p) : "memory");
+    return v;
+}
+
 // Per-row constants of the quantizer: scale, 1 / scale, zero-point and the clamp range [-z, maxq - z] of rint(w / s)
 // (clamping that integer is the same as clamping the code to [0, maxq], because the zero-point is an integer).
 struct RowGrid {
@@ -273,7 +279,10 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         if (live) {
                             double* dst = prm.E + (int64_t)row * n + p0 + 8 * m;
 #pragma unroll
-                            for (int c = 0; c < 8; ++c) v[c] *= rdiag[8 * m + c];
+                            for (int c = 0; c < 8; ++c) {
+                                v[c] *= rdiag[8 * m + c];
+                                v[c] = v[c] == v[c] ? v[c] : 0.0;        // E starts out as NaN = "not there yet"
+                            }
                             if (prm.vec16 && p0 + 8 * m + 8 <= n) {
 #pragma unroll
                                 for (int c = 0; c < 8; c += 2)
@@ -362,33 +371,34 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 #pragma unroll
                 for (int a = 0; a < 4; ++a) prod[a][0] = prod[a][1] = 0.0;
                 bool ok = true;
-                unsigned seen = 0;
 #pragma unroll
                 for (int m = 0; m <= 8; ++m) {
                     if (m < 8) {
-                        if (seen < (unsigned)(8 * b + m + 1)) {      // poll only when the last look was not enough
-                            if (lane == 0) {
-                                const long long t0 = clock64();
-                                unsigned it = 0;
-                                while ((seen = ld_acquire_u32(&prm.flags[g])) < (unsigned)(8 * b + m + 1)) {
-                                    if ((++it & 63u) == 0u) {
-                                        if (ld_acquire_u32(abort_word) != 0u) { ok = false; break; }
-                                        if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); ok = false; break; }
-                                    }
+                        // E is NaN until written: the operand of piece m is read again and again until none of this
+                        // warp's values is NaN any more, which needs neither the publisher's fence nor its counter
+                        // (those serve the CTAs that pick E up later, off the critical path).  Bounded.
+                        const long long t0 = clock64();
+                        unsigned it = 0;
+                        while (true) {
+                            bool have = true;
+#pragma unroll
+                            for (int s4 = 0; s4 < 2; ++s4)
+#pragma unroll
+                                for (int a = 0; a < 4; ++a) {
+                                    const int r = r0 + 8 * a + lq;
+                                    const double x =
+                                        r < rows ? ld_relaxed_f64(prm.E + (int64_t)r * n + p0 + 8 * m + 4 * s4 + lr) : 0.0;
+                                    af[m & 1][s4][a] = x;
+                                    have = have && x == x;
                                 }
-                                __threadfence();
+                            if (__all_sync(0xffffffffu, have)) break;
+                            if ((++it & 15u) == 0u) {
+                                bool bad = ld_acquire_u32(abort_word) != 0u;
+                                if (!bad && clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); bad = true; }
+                                if (__any_sync(0xffffffffu, bad)) { ok = false; break; }
                             }
-                            seen = __shfl_sync(0xffffffffu, seen, 0);
-                            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-                            if (!ok) break;
                         }
-#pragma unroll
-                        for (int s4 = 0; s4 < 2; ++s4)
-#pragma unroll
-                            for (int a = 0; a < 4; ++a) {
-                                const int r = r0 + 8 * a + lq;
-                                af[m & 1][s4][a] = r < rows ? __ldcg(prm.E + (int64_t)r * n + p0 + 8 * m + 4 * s4 + lr) : 0.0;
-                            }
+                        if (!ok) break;
                     }
                     if (m > 0) {
 #pragma unroll
@@ -512,6 +522,8 @@ inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p
     }
     const int groups = cdiv(rows, kSweepRows);
     if (cudaMemsetAsync(flags, 0, ((size_t)groups + 1) * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
+    // every byte 0xFF is a NaN: "not published yet" for the owner of the next block, which polls the values themselves
+    if (cudaMemsetAsync(E, 0xFF, (size_t)rows * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     SweepParams prm;
     prm.Wp = Wp; prm.U = U; prm.E = E; prm.codes_p = codes_p; prm.scale = scale; prm.zero = zero;
     prm.rows = rows; prm.n = n; prm.bits = bits;
