@@ -39,9 +39,9 @@ INT8_OVER_BF16 = 2.0                                   # nominal dense 4.5 / 2.2
 # profiles/, on the bench workload (Gram: scaled from the 16384-column capture by the calibration columns processed).
 # Each entry names the kernel sources it was taken with; when they have changed since, the traffic is reported as null.
 NCU_TRAFFIC = {
-    "chol_coop": {"bytes_per_launch": (42.40e6 + 5.05e6 + 21.75e6 + 0.77e6) / 2, "sources": ["chol.cuh", "dgemm.cuh"],
-                  "sha256_16": "ad6b456de9354004"},
-    "sweep_coop": {"bytes_per_launch": 26.26e6 + 0.0e6, "sources": ["colloop.cuh"], "sha256_16": "962d37ad9ecbf441"},
+    "chol_coop": {"bytes_per_launch": (42.40e6 + 4.33e6 + 21.75e6 + 1.04e6) / 2, "sources": ["chol.cuh", "dgemm.cuh"],
+                  "sha256_16": "94ab96d7a3238342"},
+    "sweep_coop": {"bytes_per_launch": 26.36e6 + 0.01e6, "sources": ["colloop.cuh"], "sha256_16": "0f794cd80fb7303a"},
     "gram_i8_tcgen05": {"bytes_per_launch": (508.4e6 + 31.1e6) * 4096 / 16384, "sources": ["gram.cuh"],
                         "sha256_16": "d0232587de830f4f"},
 }
