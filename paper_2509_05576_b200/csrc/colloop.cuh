@@ -214,6 +214,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
         rg.hi = maxq - rg.zp;
         int lazy = 0;
         bool prepared = false;           // Us / rdiag / blk already hold the block about to be quantized
+        bool ahead = false;              // blk holds this CTA's next block with E of the block before last folded in
         // the block being quantized: fragment a = rows 8 a + lq, columns 8 warp + 2 lr + {0, 1}
         double blk[4][2];
         for (int b = 0; b < nb; ++b) {
@@ -221,12 +222,22 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
             const int kb = n - p0 < kNB ? n - p0 : kNB;
             const bool mine = (b % cpg) == ci;
             const bool next_mine = cpg > 1 && b + 1 < nb && ((b + 1) % cpg) == ci;
+            // With four or more CTAs in the group, the owner of block b + 2 folds E[:, b] into that block while block b
+            // is still being quantized, just as the owner of block b + 1 does: the deferred update of a block by the two
+            // blocks before it then never waits for the group's counter, which is what used to delay its owner.
+            const bool next2_mine = cpg >= 4 && b + 2 < nb && ((b + 2) % cpg) == ci;
+            if (next2_mine) {
+                __syncthreads();
+                sweep_load_tile(Bb, kSweepLd, prm.U, n, p0, p0 + 2 * kNB, kNB, kNB, n, n, prm.vec16);
+                cp_async_commit();
+                load_diag(b + 2);            // nothing of it depends on E: out of the way two blocks early
+            }
             if (next_mine) {
                 // block b + 1 is quantized here next: what does not depend on E[:, b] is fetched before waiting for it
                 __syncthreads();
                 sweep_load_tile(Bb, kSweepLd, prm.U, n, p0, p0 + kNB, kNB, kNB, n, n, prm.vec16);
                 cp_async_commit();
-                load_diag(b + 1);
+                if (!ahead) load_diag(b + 1);
             }
             if (mine) {
                 // ------------------------------------------------------------ quantize block b
@@ -306,7 +317,10 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                                         if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); break; }
                                     }
                                 }
-                                atomicExch(&prm.flags[g], (unsigned)(8 * b + m + 1));
+                                // a reduction without a return value: the warp does not wait for the round trip, and
+                                // should two of them overtake each other on the way the maximum is still right (the
+                                // data of the earlier piece was fenced before its warp let this one pass)
+                                atomicMax(&prm.flags[g], (unsigned)(8 * b + m + 1));
                                 *s_pub = 8 * b + m + 1;
                             }
                         }
@@ -329,7 +343,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                     if (r0 + r < rows && c < kb) prm.codes_p[(int64_t)(r0 + r) * n + p0 + c] = Cs[r * (kNB + 4) + c];
                 }
                 prepared = false;
-            } else if (!next_mine) {
+            } else if (!next_mine && !next2_mine) {
                 // ------------------------------------------------------------ wait for all of E[:, b]
                 if (tid == 0) {
                     const long long t0 = clock64();
@@ -353,17 +367,25 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
             }
             if (b + 1 >= nb) break;
             // ---------------------------------------------------------------- deferred Eq. 11 on the owned blocks
-            if (next_mine) {
-                // block b + 1 only, straight into the fragments the chain starts from; the other blocks catch up later
+            if (next_mine || next2_mine) {
+                // block b + 1 (or b + 2) only, straight into the fragments the chain starts from; the other blocks catch
+                // up later
+                if (!(next_mine && ahead)) {
+                    const int c0 = p0 + (next_mine ? kNB : 2 * kNB);
 #pragma unroll
-                for (int a = 0; a < 4; ++a)
+                    for (int a = 0; a < 4; ++a)
 #pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const int r = r0 + 8 * a + lq, c = p0 + kNB + 8 * warp + 2 * lr + e;
-                        blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
-                    }
+                        for (int e = 0; e < 2; ++e) {
+                            const int r = r0 + 8 * a + lq, c = c0 + 8 * warp + 2 * lr + e;
+                            blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
+                        }
+                }
+                // whatever of E[:, b] is out already comes in one go through shared memory (an owner that arrives late
+                // would otherwise pay one L2 round trip per piece); the pieces still missing there are polled below
+                sweep_load_tile(Ea, kSweepLd, prm.E, n, r0, p0, kSweepRows, kNB, rows, n, prm.vec16);
+                cp_async_commit();
                 cp_async_wait<0>();
-                __syncthreads();             // U[b, b + 1] is in Bb
+                __syncthreads();             // U[b, b + 1] (or U[b, b + 2]) is in Bb, the snapshot of E[:, b] in Ea
                 // E[:, b] arrives eight columns at a time.  Every warp polls the group's counter for itself (bounded),
                 // requests the operand of piece m straight from global memory as soon as it is out, and meanwhile
                 // multiplies piece m - 1, whose operand was requested one piece earlier.
@@ -377,9 +399,18 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         // E is NaN until written: the operand of piece m is read again and again until none of this
                         // warp's values is NaN any more, which needs neither the publisher's fence nor its counter
                         // (those serve the CTAs that pick E up later, off the critical path).  Bounded.
+                        bool snap = true;
+#pragma unroll
+                        for (int s4 = 0; s4 < 2; ++s4)
+#pragma unroll
+                            for (int a = 0; a < 4; ++a) {
+                                const double x = Ea[(8 * a + lq) * kSweepLd + 8 * m + 4 * s4 + lr];
+                                af[m & 1][s4][a] = x;
+                                snap = snap && x == x;
+                            }
                         const long long t0 = clock64();
                         unsigned it = 0;
-                        while (true) {
+                        while (!__all_sync(0xffffffffu, snap)) {
                             bool have = true;
 #pragma unroll
                             for (int s4 = 0; s4 < 2; ++s4)
@@ -418,7 +449,8 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                     blk[a][0] -= prod[a][0];
                     blk[a][1] -= prod[a][1];
                 }
-                prepared = true;
+                prepared = next_mine;
+                ahead = !next_mine;
                 continue;
             }
             const int b_first = b + 1 + (((ci - (b + 1)) % cpg) + cpg) % cpg;     // first owned block beyond b
