@@ -4,6 +4,7 @@
     python -m paper_2509_05576_b200.layer_set_run --config 4 --bits 8   # the YOLOv5s-shaped stack
     python -m paper_2509_05576_b200.layer_set_run --config 5 --bits 4   # square / wide scaling shapes
     python -m paper_2509_05576_b200.layer_set_run --config 6            # ResNet-18-shaped (7: ResNet-34-shaped)
+    python -m paper_2509_05576_b200.layer_set_run --config 3 --score-mode none   # the ordering ablation (Sec. 6)
 
 Every layer goes through the five C-ABI calls (Hessian, damped inverse, grid, scores + order, sweep); each call is
 bracketed by CUDA events on the launching stream, an L2-sized buffer is rewritten before every timed repetition.
@@ -24,6 +25,8 @@ from . import ptq
 from . import workloads as wl
 
 FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
+SCORE_MODES = {"qerr": ptq.SCORE_QERR, "prune": ptq.SCORE_PRUNE, "err": ptq.SCORE_ERR, "w": ptq.SCORE_W,
+               "none": ptq.SCORE_NONE}
 INT8_OVER_BF16 = 2.0
 
 
@@ -53,6 +56,8 @@ def main(argv=None):
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--limit", type=int, default=0, help="only the first LIMIT layers (0: all)")
     ap.add_argument("--max-cols", type=int, default=0, help="skip layers with more columns (0: none)")
+    ap.add_argument("--score-mode", default="qerr", choices=sorted(SCORE_MODES),
+                    help="column ordering: qerr (Eq. 10, the method's), prune (Eq. 8), err, w, none (no sorting)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise RuntimeError("layer_set_run needs a CUDA device")
@@ -72,7 +77,7 @@ def main(argv=None):
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
     ws = ptq.Workspace()
     rows_out = []
-    totals = {"weights": 0, "ms": 0.0}
+    totals = {"weights": 0, "ms": 0.0, "loss": 0.0}
     stage_tot = {}
     print(f"{'layer':28s} {'rows':>5s} {'cols':>6s} {'n':>5s} {'b':>2s} {'total ms':>9s} {'Mw/s':>8s} "
           f"{'hess':>7s} {'inv':>7s} {'order':>6s} {'sweep':>7s} {'%int8':>6s} {'%f64 inv':>8s} {'%f64 swp':>8s} {'loss':>12s}")
@@ -80,14 +85,15 @@ def main(argv=None):
         W, X = wl.make_layer(spec)
         Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
         bufs = ptq.LayerBuffers(spec.rows, spec.cols)
-        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, bufs=bufs, ws=ws, stream=s)    # warm-up
+        mode = SCORE_MODES[args.score_mode]
+        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=mode, bufs=bufs, ws=ws, stream=s)    # warm-up
         torch.cuda.synchronize()
         ptq.check_status(bufs.status, spec.name)
         per = {}
         for rep in range(args.reps):
             flush.fill_(rep)
             ev = []
-            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, bufs=bufs, ws=ws, stream=s, events=ev)
+            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=mode, bufs=bufs, ws=ws, stream=s, events=ev)
             torch.cuda.synchronize()
             for name, a, b in ev:
                 per.setdefault(name, []).append(a.elapsed_time(b))
@@ -107,10 +113,12 @@ def main(argv=None):
                          "ms": total, "stages_ms": st, "roofline_frac": frac, "loss": loss})
         totals["weights"] += spec.weights
         totals["ms"] += total
+        totals["loss"] += loss
         for k, v in st.items():
             stage_tot[k] = stage_tot.get(k, 0.0) + v
         del Wd, Xd, bufs
-    print(json.dumps({"config": args.config, "layers": len(rows_out), "weights": totals["weights"],
+    print(json.dumps({"config": args.config, "score_mode": args.score_mode, "loss_sum": totals["loss"],
+                      "layers": len(rows_out), "weights": totals["weights"],
                       "total_ms": totals["ms"], "weights_per_s": totals["weights"] / (totals["ms"] * 1e-3),
                       "stage_total_ms": stage_tot, "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak,
                                                              "fp64_tflops": FP64_PEAK_TFLOPS, "source": src}}))
