@@ -190,7 +190,9 @@ def algorithmic_work(spec):
     return {
         "gram_i8_tcgen05": ("tensor", c * (c + 1) * n),            # symmetric half of 2 X X^T
         "gram_split": ("hbm", 4.0 * c * n + 6.0 * c * n),           # reads X once, writes six int8 planes
-        "chol_coop": ("alu", 2 * (c ** 3 / 3.0)),                   # two Cholesky factorisations, c^3/3 flops each
+        # two launches: Cholesky of H + lambda I together with the inverse of its factor (c^3/3 + c^3/3, Sec. 5 item 1),
+        # and the Cholesky of the permuted inverse Hessian (c^3/3, the blocked form of Eq. 12)
+        "chol_coop": ("alu", 3 * (c ** 3 / 3.0)),
         "dgemm_lauum": ("alu", c ** 3 / 3.0),
         "dgemm_loss": ("alu", 1.0 * r * c * c),                     # H symmetric: half of the 2 r c^2 of the plain product
         # sweep: float64 W in and E out, codes out, the upper factor U once per 32-row group is NOT counted (L2)
