@@ -36,6 +36,28 @@ def test_hessian_matches_oracle(cols, n, f64):
     assert np.max(np.abs(Hn - ref)) <= 2e-12 * np.max(np.abs(ref))
 
 
+def test_hessian_sliced_last_wave_and_two_launches_per_call():
+    """1600 columns are 169 output tiles: one full wave of the persistent grid and a last wave whose tiles are cut
+    along the calibration length; 17000 calibration columns make the call two launches (16384 + 616).  The sliced
+    tiles must come out exactly as whole ones would: compared with the oracle and, bit for bit, with the same call on
+    a matrix whose tile count leaves no partial wave to slice (the first 1280 columns: 110 tiles, more than half a wave)."""
+    cols, n = 1600, 17000
+    _, X = _layer(4, cols, n, 4242)
+    ref = oracle.hessian_accumulate(X)
+    st, ws = ptq.new_status(), ptq.Workspace()
+    H = torch.zeros((cols, cols), dtype=torch.float64, device="cuda")
+    ptq.hessian_accumulate(H, _cuda(X), ws, st)
+    sub = 1280
+    Hs = torch.zeros((sub, sub), dtype=torch.float64, device="cuda")
+    ptq.hessian_accumulate(Hs, _cuda(X[:sub]), ws, st)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    Hn = H.cpu().numpy()
+    assert np.array_equal(Hn, Hn.T)
+    assert np.max(np.abs(Hn - ref)) <= 2e-12 * np.max(np.abs(ref))
+    assert np.array_equal(Hs.cpu().numpy(), Hn[:sub, :sub])
+
+
 @pytest.mark.parametrize("xdist", ["normal", "silu", "halfnormal_sparse30"])
 def test_hessian_signed_and_sparse_inputs_accumulate_in_chunks(xdist):
     cols, n = 190, 768
