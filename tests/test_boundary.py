@@ -83,3 +83,30 @@ def test_binding_refuses_cpu_tensors(lib):
     from paper_2509_05576_b200 import ptq
     with pytest.raises(ValueError):
         ptq.hessian_accumulate(torch.zeros(4, 4, dtype=torch.float64), torch.zeros(4, 8), None, None)
+
+
+def test_layer_shape_sets_have_the_published_weight_counts():
+    """The synthetic layer sets take nothing but shapes from the networks of Sec. 6: their weight totals are the
+    well-known convolution + classifier weight counts of those architectures."""
+    from paper_2509_05576_b200 import workloads as wl
+    assert sum(r * c for _, r, c in wl.resnet50_shapes()) == 25_502_912 and len(wl.resnet50_shapes()) == 54
+    assert sum(r * c for _, r, c in wl.resnet_basic_shapes((2, 2, 2, 2))) == 11_678_912      # ResNet-18
+    assert sum(r * c for _, r, c in wl.resnet_basic_shapes((3, 4, 6, 3))) == 21_779_648      # ResNet-34
+    assert sum(r * c for _, r, c in wl.yolov5s_shapes()[:-1]) == 7_215_616
+    for spec in wl.conv_cases() + wl.resnet_conv_specs():
+        oh, ow = spec.out_hw
+        assert oh >= 1 and ow >= 1 and spec.n == spec.batch * oh * ow and spec.cols == spec.channels * spec.kh * spec.kw
+    # the convolution whose unfolded input is the benchmark layer's shape
+    c = wl.resnet_conv_specs()[0]
+    assert (c.out_channels, c.cols) == (256, 2304) and abs(c.n - 4096) < 64
+
+
+def test_conv_entry_point_rejects_bad_arguments_without_a_gpu(lib):
+    from paper_2509_05576_b200 import ptq
+    fake = ctypes.c_void_p(4096)
+    f = lib.ptq_hessian_accumulate_conv
+    assert f(fake, fake, 1, 3, 8, 8, 3, 3, 0, 1, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG      # stride 0
+    assert f(fake, fake, 1, 3, 8, 8, 12, 3, 1, 1, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG     # kernel > image
+    assert f(None, fake, 1, 3, 8, 8, 3, 3, 1, 1, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG
+    assert f(fake, fake, 1, 3, 8, 8, 3, 3, 1, 1, fake, 16, fake, None) == ptq.ERR_WORKSPACE
+    assert f(fake, fake, 1, 1 << 18, 8, 8, 3, 3, 1, 1, fake, 1 << 40, fake, None) == ptq.ERR_UNSUPPORTED   # cols > 2^20
