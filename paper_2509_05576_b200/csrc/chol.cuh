@@ -495,33 +495,42 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
             }
             return pc;
         };
-        auto load_piece = [&](const Piece& pc, int stg) {
-            double* dst = opnd + stg * 2 * kNB * kCholLd;
-            chol_load_block(dst, A, ld, n, k0, pc.i0, lgH, vec16);                      // U[k0 + kk][i0 + r]
-            chol_load_block(dst + kNB * kCholLd, pc.Bsrc, ld, n, k0, pc.j0, 6, vec16);  // U or W [k0 + kk][j0 + c]
-        };
-        int stage = 0;
+        // Operand blocks: slot s of the A half holds U[k][i-block] (as[kk][r]), slot s of the B half U or W [k][j-block].
+        // Every CTA takes a contiguous run of the list, in which consecutive tiles mostly share their row block: the A
+        // operand then stays where it is and only B is fetched.
+        double* abuf = opnd;                                  // [2][64][kCholLd]
+        double* bbuf = opnd + 2 * kNB * kCholLd;              // [2][64][kCholLd]
+        const int per = (TP + Gt - 1) / Gt;
+        const int tp_beg = me * per, tp_end = tp_beg + per < TP ? tp_beg + per : TP;
+        int stage = 0, a_slot = 0, a_next = 0;
         Piece cur{}, nxt{};
-        if (me < TP) {
-            cur = piece_of(me);
-            load_piece(cur, 0);
+        if (tp_beg < tp_end) {
+            cur = piece_of(tp_beg);
+            chol_load_block(abuf, A, ld, n, k0, cur.i0, lgH, vec16);
+            chol_load_block(bbuf, cur.Bsrc, ld, n, k0, cur.j0, 6, vec16);
         }
         cp_async_commit();
-        for (int tp = me; tp < TP; tp += Gt) {
-            if (tp + Gt < TP) {
-                nxt = piece_of(tp + Gt);
-                load_piece(nxt, stage ^ 1);
+        for (int tp = tp_beg; tp < tp_end; ++tp) {
+            if (tp + 1 < tp_end) {
+                nxt = piece_of(tp + 1);
+                a_next = a_slot;
+                if (nxt.i0 != cur.i0) {
+                    a_next = a_slot ^ 1;
+                    chol_load_block(abuf + a_next * kNB * kCholLd, A, ld, n, k0, nxt.i0, lgH, vec16);
+                }
+                chol_load_block(bbuf + (stage ^ 1) * kNB * kCholLd, nxt.Bsrc, ld, n, k0, nxt.j0, 6, vec16);
             }
             cp_async_commit();
             cp_async_wait<1>();
             __syncthreads();
-            const double* as = opnd + stage * 2 * kNB * kCholLd;
-            const double* bs = as + kNB * kCholLd;
+            const double* as = abuf + a_slot * kNB * kCholLd;
+            const double* bs = bbuf + stage * kNB * kCholLd;
             if (lgH == 6) chol_trailing_piece<64>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
             else if (lgH == 5) chol_trailing_piece<32>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
             else chol_trailing_piece<16>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
-            __syncthreads();     // all warps are done with this stage before it is refilled
+            __syncthreads();     // all warps are done with these operands before their slots are refilled
             stage ^= 1;
+            a_slot = a_next;
             cur = nxt;
         }
         cp_async_wait<0>();
