@@ -375,6 +375,21 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int6
     // hides behind it
     double old[FM][FN][2], acc[FM][FN][2];
     bool keep[FM][FN][2];
+    // a piece inside the matrix and off the diagonal needs no bounds or triangle tests at all
+    const bool plain = vec16 && tri_off < 0 && i0 + H <= n && j0 + kNB <= n;
+    if (plain) {
+        const double* src = C + (int64_t)(i0 + wm0 + lq) * ld + j0 + wn0 + 2 * lr;
+#pragma unroll
+        for (int a = 0; a < FM; ++a)
+#pragma unroll
+            for (int b = 0; b < FN; ++b) {
+                const double2 v = __ldcg(reinterpret_cast<const double2*>(src + (int64_t)(8 * a) * ld + 8 * b));
+                old[a][b][0] = v.x;
+                old[a][b][1] = v.y;
+                acc[a][b][0] = acc[a][b][1] = 0.0;
+                keep[a][b][0] = keep[a][b][1] = true;
+            }
+    } else
 #pragma unroll
     for (int a = 0; a < FM; ++a) {
         const int r = wm0 + a * 8 + lq;
@@ -407,6 +422,16 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int6
         for (int a = 0; a < FM; ++a)
 #pragma unroll
             for (int b = 0; b < FN; ++b) dmma_884(acc[a][b][0], acc[a][b][1], af[a], bf[b]);
+    }
+    if (plain) {
+        double* dst = C + (int64_t)(i0 + wm0 + lq) * ld + j0 + wn0 + 2 * lr;
+#pragma unroll
+        for (int a = 0; a < FM; ++a)
+#pragma unroll
+            for (int b = 0; b < FN; ++b)
+                __stcg(reinterpret_cast<double2*>(dst + (int64_t)(8 * a) * ld + 8 * b),
+                       make_double2(old[a][b][0] - acc[a][b][0], old[a][b][1] - acc[a][b][1]));
+        return;
     }
 #pragma unroll
     for (int a = 0; a < FM; ++a) {
