@@ -98,13 +98,17 @@ __device__ __forceinline__ void cp_async16_cg(void* smem_dst, const void* gsrc, 
 // Loads the 64 x ncols block A[r0 .. r0+63][c0 .. c0+ncols-1] into dst[64][kCholLd], ncols = 1 << lg in {16, 32, 64};
 // entries beyond n are zero.  Every thread copies a fixed column (pair) of successive row groups, so a block that lies
 // inside the matrix needs one pointer increment per copy and no bounds test.
+// NT threads take part (the first NT of the CTA): all of them, or the first four warps when the other four are to
+// go on computing meanwhile.
+template <int NT = kCholThreads>
 __device__ __forceinline__ void chol_load_block(double* dst, const double* __restrict__ A, int64_t ld, int n, int r0,
                                                 int c0, int lg, int vec16) {
+    if (NT < kCholThreads && threadIdx.x >= NT) return;
     const bool interior = r0 + kNB <= n && c0 + (1 << lg) <= n;
     if (vec16) {
         const int sh = lg - 1;                           // pairs per row = 1 << sh
         const int c = (threadIdx.x & ((1 << sh) - 1)) * 2;
-        const int rstep = kCholThreads >> sh;
+        const int rstep = NT >> sh;
         int r = threadIdx.x >> sh;
         const double* src = A + (int64_t)(r0 + r) * ld + c0 + c;
         double* d = dst + r * kCholLd + c;
@@ -118,7 +122,7 @@ __device__ __forceinline__ void chol_load_block(double* dst, const double* __res
         }
     } else {
         const int c = threadIdx.x & ((1 << lg) - 1);
-        const int rstep = kCholThreads >> lg;
+        const int rstep = NT >> lg;
         int r = threadIdx.x >> lg;
         const double* src = A + (int64_t)(r0 + r) * ld + c0 + c;
         double* d = dst + r * kCholLd + c;
@@ -536,24 +540,27 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         }
         cp_async_commit();
         for (int tp = tp_beg; tp < tp_end; ++tp) {
+            cp_async_wait<0>();
+            __syncthreads();         // this tile's operands have landed; the slots of the tile before are free
+            // The next tile's operands are requested by the first four warps only: the copies keep the issuing warps
+            // busy for several hundred cycles, during which the other four (one per scheduler) already feed the
+            // tensor pipe.
             if (tp + 1 < tp_end) {
                 nxt = piece_of(tp + 1);
                 a_next = a_slot;
                 if (nxt.i0 != cur.i0) {
                     a_next = a_slot ^ 1;
-                    chol_load_block(abuf + a_next * kNB * kCholLd, A, ld, n, k0, nxt.i0, lgH, vec16);
+                    chol_load_block<kCholThreads / 2>(abuf + a_next * kNB * kCholLd, A, ld, n, k0, nxt.i0, lgH, vec16);
                 }
-                chol_load_block(bbuf + (stage ^ 1) * kNB * kCholLd, nxt.Bsrc, ld, n, k0, nxt.j0, 6, vec16);
+                chol_load_block<kCholThreads / 2>(bbuf + (stage ^ 1) * kNB * kCholLd, nxt.Bsrc, ld, n, k0, nxt.j0, 6,
+                                                  vec16);
             }
             cp_async_commit();
-            cp_async_wait<1>();
-            __syncthreads();
             const double* as = abuf + a_slot * kNB * kCholLd;
             const double* bs = bbuf + stage * kNB * kCholLd;
             if (lgH == 6) chol_trailing_piece<64>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
             else if (lgH == 5) chol_trailing_piece<32>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
             else chol_trailing_piece<16>(cur.C, ld, n, as, bs, cur.i0, cur.j0, cur.tri, vec16);
-            __syncthreads();     // all warps are done with these operands before their slots are refilled
             stage ^= 1;
             a_slot = a_next;
             cur = nxt;
