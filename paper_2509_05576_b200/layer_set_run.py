@@ -56,6 +56,9 @@ def main(argv=None):
     ap.add_argument("--reps", type=int, default=2)
     ap.add_argument("--limit", type=int, default=0, help="only the first LIMIT layers (0: all)")
     ap.add_argument("--max-cols", type=int, default=0, help="skip layers with more columns (0: none)")
+    ap.add_argument("--streams", type=int, default=1,
+                    help="> 1: also run the whole set with the layers dealt round-robin onto this many streams "
+                         "(inputs resident, nothing synchronised in between) and report the wall time of that")
     ap.add_argument("--score-mode", default="qerr", choices=sorted(SCORE_MODES),
                     help="column ordering: qerr (Eq. 10, the method's), prune (Eq. 8), err, w, none (no sorting)")
     args = ap.parse_args(argv)
@@ -117,7 +120,47 @@ def main(argv=None):
         for k, v in st.items():
             stage_tot[k] = stage_tot.get(k, 0.0) + v
         del Wd, Xd, bufs
+    overlapped = None
+    if args.streams > 1:
+        # independent layers on several streams: every stream has its own workspace and output buffers; the inputs
+        # of all layers are put on the device first; one event pair around the whole set
+        data = []
+        for spec in specs:
+            W, X = wl.make_layer(spec)
+            data.append((spec, torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()))
+        outs = [ptq.LayerBuffers(spec.rows, spec.cols) for spec in specs]      # one set of outputs per layer, kept
+        streams = [torch.cuda.Stream() for _ in range(args.streams)]
+        wss = [ptq.Workspace() for _ in streams]
+
+        def run_set():
+            for i, (spec, Wd, Xd) in enumerate(data):
+                k = i % len(streams)
+                ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=SCORE_MODES[args.score_mode],
+                                        bufs=outs[i], ws=wss[k], stream=streams[k])
+
+        times = []
+        for rep in range(args.reps + 1):
+            torch.cuda.synchronize()
+            flush.fill_(rep)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(s)
+            for st_ in streams:
+                st_.wait_stream(s)
+            run_set()
+            for st_ in streams:
+                s.wait_stream(st_)
+            e1.record(s)
+            torch.cuda.synchronize()
+            if rep > 0:
+                times.append(e0.elapsed_time(e1))
+        for o, spec in zip(outs, specs):
+            ptq.check_status(o.status, spec.name)
+        overlapped = {"streams": args.streams, "set_ms": float(np.median(times)),
+                      "loss_sum": float(sum(o.loss.item() for o in outs))}
+        print(f"whole set on {args.streams} streams: {overlapped['set_ms']:.2f} ms "
+              f"(sum of the per-layer times on one stream: {totals['ms']:.2f} ms)")
     print(json.dumps({"config": args.config, "score_mode": args.score_mode, "loss_sum": totals["loss"],
+                      "overlapped": overlapped,
                       "layers": len(rows_out), "weights": totals["weights"],
                       "total_ms": totals["ms"], "weights_per_s": totals["weights"] / (totals["ms"] * 1e-3),
                       "stage_total_ms": stage_tot, "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak,
