@@ -23,6 +23,7 @@ _LIB = os.path.join(_HERE, "liboracle.so")
 OK, ERR_INVALID_ARG, ERR_NOT_SPD, ERR_NOMEM = 0, 1, 4, 9
 DAMP_REL_MEAN_DIAG, DAMP_ABS = 0, 1
 SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
+SCORE_ASCENDING = 16          # added to a score mode: sort by S ascending (the "asc" keys of Sec. 4.1)
 
 
 class OracleError(RuntimeError):
@@ -64,6 +65,12 @@ def lib():
         L.oracle_quantize_layer_ex.argtypes = [pf, c_int, c_int, c_int64, pd, pi, pf, pf, c_int, pu, pf,
                                                pd, pd, pu, pd, pd, pd, pd]
         L.oracle_loss_direct.argtypes = [pf, pf, c_int, c_int, c_int64, c_int64, pf, c_int, c_int64]
+        L.oracle_factor_upper.argtypes = [pd, pi, c_int, pd, POINTER(c_int)]
+        L.oracle_quantize_rows_factor.argtypes = [pf, c_int, c_int, c_int64, pd, pi, pf, pf, c_int, pu, pf, pd]
+        L.oracle_quantize_layer_dynamic.argtypes = [pf, c_int, c_int, c_int64, pd, pf, pf, c_int, c_int, c_int, pu,
+                                                    pf, pi, pd, pd, pd]
+        L.oracle_quantize_layer_per_row.argtypes = [pf, c_int, c_int, c_int64, pd, pd, pf, pf, c_int, c_int, pu, pf,
+                                                    pi, pd, pd]
         L.oracle_loss_direct.restype = c_double
         _lib = L
     return _lib
@@ -200,6 +207,97 @@ def quantize_layer(W, Hinv, perm, scale, zero, bits, H_undamped=None, forced_cod
         out["prer"] = prer
     if want_trace:
         out["A_trace"], out["W_trace"] = A_tr, W_tr
+    return out
+
+
+def factor_upper(Hinv, perm):
+    """U with Hinv[perm][:, perm] = U^T U (upper triangular), by the oracle's own plain Cholesky."""
+    Hinv = np.ascontiguousarray(Hinv, dtype=np.float64)
+    perm = np.ascontiguousarray(perm, dtype=np.int32)
+    cols = Hinv.shape[0]
+    U = np.empty((cols, cols), dtype=np.float64)
+    info = c_int(-1)
+    st = lib().oracle_factor_upper(_p(Hinv, c_double), _p(perm, c_int32), cols, _p(U, c_double), ctypes.byref(info))
+    if st:
+        raise OracleError(st, "factor_upper", info.value)
+    return U
+
+
+def quantize_rows_factor(W, U, perm, scale, zero, bits, want_prer=False):
+    """The column loop in factor form (e = (w - q) / U_pp, w_j -= e U_pj) on the given rows.  Licensed by its pin
+    against the literal Eq. 11 / Eq. 12 loop; for layers too wide for that loop."""
+    W = _f32(W)
+    rows, cols = W.shape
+    U = np.ascontiguousarray(U, dtype=np.float64)
+    perm = np.ascontiguousarray(perm, dtype=np.int32)
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    zero = np.ascontiguousarray(zero, dtype=np.float32)
+    codes = np.empty((rows, cols), dtype=np.uint8)
+    What = np.empty((rows, cols), dtype=np.float32)
+    prer = np.empty((rows, cols), dtype=np.float64) if want_prer else None
+    st = lib().oracle_quantize_rows_factor(_p(W, c_float), rows, cols, W.strides[0] // 4, _p(U, c_double),
+                                           _p(perm, c_int32), _p(scale, c_float), _p(zero, c_float), int(bits),
+                                           _p(codes, c_uint8), _p(What, c_float), _p(prer, c_double))
+    if st:
+        raise OracleError(st, "quantize_rows_factor")
+    out = {"codes": codes, "What": What}
+    if want_prer:
+        out["prer"] = prer
+    return out
+
+
+def quantize_layer_dynamic(W, Hinv, scale, zero, bits, block, mode=SCORE_QERR, H_undamped=None, want_prer=False):
+    """Dynamic re-ranking (Sec. 5): the remaining columns are re-scored from the current weights and the current
+    inverse Hessian every `block` columns.  Returns codes, What, order (the sequence of columns) and the extras."""
+    W = _f32(W)
+    rows, cols = W.shape
+    Hinv = np.ascontiguousarray(Hinv, dtype=np.float64)
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    zero = np.ascontiguousarray(zero, dtype=np.float32)
+    codes = np.empty((rows, cols), dtype=np.uint8)
+    What = np.empty((rows, cols), dtype=np.float32)
+    order = np.empty(cols, dtype=np.int32)
+    Hu = None if H_undamped is None else np.ascontiguousarray(H_undamped, dtype=np.float64)
+    loss = c_double(float("nan"))
+    prer = np.empty((rows, cols), dtype=np.float64) if want_prer else None
+    st = lib().oracle_quantize_layer_dynamic(_p(W, c_float), rows, cols, W.strides[0] // 4, _p(Hinv, c_double),
+                                             _p(scale, c_float), _p(zero, c_float), int(bits), int(mode), int(block),
+                                             _p(codes, c_uint8), _p(What, c_float), _p(order, c_int32),
+                                             _p(Hu, c_double), ctypes.byref(loss) if Hu is not None else None,
+                                             _p(prer, c_double))
+    if st:
+        raise OracleError(st, "quantize_layer_dynamic")
+    out = {"codes": codes, "What": What, "order": order}
+    if Hu is not None:
+        out["loss"] = loss.value
+    if want_prer:
+        out["prer"] = prer
+    return out
+
+
+def quantize_layer_per_row(W, Hinv, Hinv_diag, scale, zero, bits, mode=SCORE_QERR, H_undamped=None):
+    """The non-parallel arm (Sec. 4.2): every row ranked by its own sensitivities and quantized against its own copy
+    of the inverse Hessian.  Returns codes, What, perm_rows [rows, cols] and the loss when H is given."""
+    W = _f32(W)
+    rows, cols = W.shape
+    Hinv = np.ascontiguousarray(Hinv, dtype=np.float64)
+    diag = None if Hinv_diag is None else np.ascontiguousarray(Hinv_diag, dtype=np.float64)
+    scale = np.ascontiguousarray(scale, dtype=np.float32)
+    zero = np.ascontiguousarray(zero, dtype=np.float32)
+    codes = np.empty((rows, cols), dtype=np.uint8)
+    What = np.empty((rows, cols), dtype=np.float32)
+    perm_rows = np.empty((rows, cols), dtype=np.int32)
+    Hu = None if H_undamped is None else np.ascontiguousarray(H_undamped, dtype=np.float64)
+    loss = c_double(float("nan"))
+    st = lib().oracle_quantize_layer_per_row(_p(W, c_float), rows, cols, W.strides[0] // 4, _p(Hinv, c_double),
+                                             _p(diag, c_double), _p(scale, c_float), _p(zero, c_float), int(bits),
+                                             int(mode), _p(codes, c_uint8), _p(What, c_float), _p(perm_rows, c_int32),
+                                             _p(Hu, c_double), ctypes.byref(loss) if Hu is not None else None)
+    if st:
+        raise OracleError(st, "quantize_layer_per_row")
+    out = {"codes": codes, "What": What, "perm_rows": perm_rows}
+    if Hu is not None:
+        out["loss"] = loss.value
     return out
 
 

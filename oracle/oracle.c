@@ -17,7 +17,9 @@
  * Pins (tests/test_oracle_pins.py): identity Hessian => round-to-nearest; every Eq. 12
  * update equals direct inversion of the remaining sub-matrix; Eq. 11 equals the constrained
  * least-squares minimiser; damped-loss sum identity; brute-force enumeration on tiny rows;
- * hand-worked ordering example; Gram / inverse against library routines.
+ * hand-worked ordering example; Gram / inverse against library routines; the factor-form mode
+ * against the literal loop and a library Cholesky; dynamic re-ranking against its definition
+ * replayed through the literal loop; the per-row mode against the hand example and single-row runs.
  * Parity unpinned: the greedy rounding decisions of a general layer have no external
  * definition beyond "nearest level of the compensated value"; they are pinned only through
  * the quantities that determine them.
@@ -32,7 +34,7 @@
 
 enum { ORACLE_OK = 0, ORACLE_ERR_INVALID_ARG = 1, ORACLE_ERR_NOT_SPD = 4, ORACLE_ERR_NOMEM = 9 };
 enum { DAMP_REL_MEAN_DIAG = 0, DAMP_ABS = 1 };
-enum { SCORE_QERR = 0, SCORE_PRUNE = 1, SCORE_ERR = 2, SCORE_W = 3, SCORE_NONE = 4 };
+enum { SCORE_QERR = 0, SCORE_PRUNE = 1, SCORE_ERR = 2, SCORE_W = 3, SCORE_NONE = 4, SCORE_ASCENDING = 16 };
 
 int oracle_version(void) { return 1; }
 
@@ -249,21 +251,29 @@ int oracle_quant_code(double w, float scale, float zero, int bits) {
  *   QERR : (w - quant(w))^2 / (2 [Hinv]_jj)       PRUNE : w^2 / (2 [Hinv]_jj)
  *   ERR  : (w - quant(w))^2                        W     : w^2
  *   NONE : S_j = 0, identity order
+ * Sec. 4.1 names every key in a descending ("des") and an ascending ("asc") variant: with
+ * SCORE_ASCENDING added to the mode the columns are sorted by S ascending instead (equal scores
+ * still keep the lower column index first).
  * ------------------------------------------------------------------------------------- */
 static const double *g_sort_keys;
-static int cmp_desc_stable(const void *pa, const void *pb) {
+static int g_sort_ascending;
+static int cmp_score_stable(const void *pa, const void *pb) {
     const int a = *(const int *)pa, b = *(const int *)pb;
     const double ka = g_sort_keys[a], kb = g_sort_keys[b];
-    if (ka > kb) return -1;
-    if (ka < kb) return 1;
+    if (ka != kb) {
+        const int a_first = g_sort_ascending ? (ka < kb) : (ka > kb);
+        return a_first ? -1 : 1;
+    }
     return (a > b) - (a < b);
 }
 
 int oracle_sensitivity_order(const float *W, int rows, int cols, int64_t ldw, const double *Hinv_diag,
-                             const float *scale, const float *zero, int bits, int mode, double *S,
-                             int32_t *perm) {
+                             const float *scale, const float *zero, int bits, int mode_and_direction,
+                             double *S, int32_t *perm) {
     if (!W || !S || !perm || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8)
         return ORACLE_ERR_INVALID_ARG;
+    const int ascending = (mode_and_direction & SCORE_ASCENDING) != 0;
+    const int mode = mode_and_direction & ~SCORE_ASCENDING;
     if (mode < 0 || mode > SCORE_NONE) return ORACLE_ERR_INVALID_ARG;
     if ((mode == SCORE_QERR || mode == SCORE_PRUNE) && !Hinv_diag) return ORACLE_ERR_INVALID_ARG;
     if ((mode == SCORE_QERR || mode == SCORE_ERR) && (!scale || !zero)) return ORACLE_ERR_INVALID_ARG;
@@ -293,7 +303,8 @@ int oracle_sensitivity_order(const float *W, int rows, int cols, int64_t ldw, co
         perm[j] = j;
     }
     g_sort_keys = S;
-    qsort(perm, (size_t)cols, sizeof(int32_t), cmp_desc_stable);
+    g_sort_ascending = ascending;
+    qsort(perm, (size_t)cols, sizeof(int32_t), cmp_score_stable);
     return ORACLE_OK;
 }
 
@@ -454,4 +465,249 @@ double oracle_loss_direct(const float *W, const float *What, int rows, int cols,
     for (int i = 0; i < rows; ++i) total += rowsum[i];
     free(rowsum);
     return total;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Factor form of the column loop, for layers too wide for the literal Eq. 12 loop (which costs
+ * cols^3 / 3 multiply-adds over a cols^2 matrix whatever the number of rows).
+ *
+ * Eq. 12 is one step of a right-looking Cholesky factorisation: with A = Hinv[perm][:, perm] = U^T U
+ * (U upper triangular), the matrix that Eq. 12 leaves before step p has row p equal to
+ * U[p][p] * U[p][p:], so Eq. 11 for column p reads
+ *     e_i = (w_ip - q_ip) / U[p][p],    w_ij -= e_i * U[p][j]   (j > p).
+ * This mode is licensed only by its pins: tests/test_oracle_pins.py shows it equal to the literal
+ * loop of oracle_quantize_layer_ex (codes, What, pre-rounding values) on every size the literal
+ * loop reaches; the literal loop stays the definition.
+ *
+ * oracle_factor_upper: A = L L^T column by column (the same plain Cholesky as in oracle_prepare_hinv,
+ * every sum in ascending index order), U[p][j] = L[j][p]; the strictly lower part of U is zero.
+ * ------------------------------------------------------------------------------------- */
+int oracle_factor_upper(const double *Hinv, const int32_t *perm, int cols, double *U, int *info) {
+    if (!Hinv || !perm || !U || cols < 1) return ORACLE_ERR_INVALID_ARG;
+    const size_t n = (size_t)cols;
+    for (size_t j = 0; j < n; ++j)
+        if (perm[j] < 0 || perm[j] >= cols) return ORACLE_ERR_INVALID_ARG;
+    double *L = (double *)calloc(n * n, sizeof(double));
+    if (!L) return ORACLE_ERR_NOMEM;
+    int bad = -1;
+    for (size_t j = 0; j < n && bad < 0; ++j) {
+        double s = Hinv[(size_t)perm[j] * n + (size_t)perm[j]];
+        for (size_t k = 0; k < j; ++k) s -= L[j * n + k] * L[j * n + k];
+        if (!(s > 0.0) || !isfinite(s)) { bad = (int)j; break; }
+        const double ljj = sqrt(s);
+        L[j * n + j] = ljj;
+#pragma omp parallel for schedule(static)
+        for (size_t i = j + 1; i < n; ++i) {
+            double t = Hinv[(size_t)perm[i] * n + (size_t)perm[j]];
+            for (size_t k = 0; k < j; ++k) t -= L[i * n + k] * L[j * n + k];
+            L[i * n + j] = t / ljj;
+        }
+    }
+    if (bad >= 0) {
+        if (info) info[0] = bad;
+        free(L);
+        return ORACLE_ERR_NOT_SPD;
+    }
+    for (size_t p = 0; p < n; ++p)
+        for (size_t j = 0; j < n; ++j) U[p * n + j] = j >= p ? L[j * n + p] : 0.0;
+    free(L);
+    return ORACLE_OK;
+}
+
+/* The sweep of Sec. 4.2 steps 4-5 on the given rows with the factor U of oracle_factor_upper.
+ * codes / What / prer as in oracle_quantize_layer_ex (original column order; What, prer may be NULL). */
+int oracle_quantize_rows_factor(const float *W, int rows, int cols, int64_t ldw, const double *U,
+                                const int32_t *perm, const float *scale, const float *zero, int bits,
+                                uint8_t *codes, float *What, double *prer) {
+    if (!W || !U || !perm || !scale || !zero || !codes || rows < 1 || cols < 1 || ldw < cols || bits < 2 ||
+        bits > 8)
+        return ORACLE_ERR_INVALID_ARG;
+    const size_t n = (size_t)cols;
+    const int maxq = (1 << bits) - 1;
+    int fail = 0;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int i = 0; i < rows; ++i) {
+        double *w = (double *)malloc(n * sizeof(double));
+        if (!w) {
+#pragma omp atomic write
+            fail = 1;
+            continue;
+        }
+        const double sc = (double)scale[i], zp = (double)zero[i];
+        for (size_t p = 0; p < n; ++p) w[p] = (double)W[(size_t)i * (size_t)ldw + (size_t)perm[p]];
+        for (size_t p = 0; p < n; ++p) {
+            const double *Up = U + p * n;
+            const size_t j0 = (size_t)perm[p];
+            if (prer) prer[(size_t)i * n + j0] = w[p] / sc;
+            const int c = quant_code(w[p], sc, zp, maxq);
+            const double q = dequant(c, sc, zp);
+            const double e = (w[p] - q) / Up[p];
+            for (size_t j = p + 1; j < n; ++j) w[j] -= e * Up[j];
+            codes[(size_t)i * n + j0] = (uint8_t)c;
+            if (What) What[(size_t)i * n + j0] = (float)q;
+        }
+        free(w);
+    }
+    return fail ? ORACLE_ERR_NOMEM : ORACLE_OK;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Dynamic re-ranking (Sec. 5 writes the sort inside the per-column loop; read literally, the
+ * columns still to be quantized are ranked again as the loop proceeds).  Every `block` columns
+ * the scores of the REMAINING columns are recomputed from the CURRENT (compensated) weights and
+ * the diagonal of the CURRENT (Eq.-12-updated) inverse Hessian, the remaining columns are sorted
+ * by them (same keys, direction and tie rule as oracle_sensitivity_order), and the next `block`
+ * columns are quantized in that order with Eq. 11 / Eq. 12 applied literally, in the original
+ * index space (no permutation of A is ever formed).  block >= cols is the static method.
+ *   order_out [cols]: the sequence in which the columns were quantized.
+ * ------------------------------------------------------------------------------------- */
+int oracle_quantize_layer_dynamic(const float *W, int rows, int cols, int64_t ldw, const double *Hinv,
+                                  const float *scale, const float *zero, int bits, int mode_and_direction,
+                                  int block, uint8_t *codes, float *What, int32_t *order_out,
+                                  const double *H_undamped, double *loss_out, double *prer) {
+    if (!W || !Hinv || !scale || !zero || !codes || !order_out || rows < 1 || cols < 1 || ldw < cols ||
+        bits < 2 || bits > 8 || block < 1)
+        return ORACLE_ERR_INVALID_ARG;
+    const int ascending = (mode_and_direction & SCORE_ASCENDING) != 0;
+    const int mode = mode_and_direction & ~SCORE_ASCENDING;
+    if (mode < 0 || mode > SCORE_NONE) return ORACLE_ERR_INVALID_ARG;
+    const size_t n = (size_t)cols, m = (size_t)rows;
+    const int maxq = (1 << bits) - 1;
+    double *A = (double *)malloc(n * n * sizeof(double));
+    double *Wc = (double *)malloc(m * n * sizeof(double));
+    double *S = (double *)malloc(n * sizeof(double));
+    double *tcol = (double *)malloc(n * sizeof(double));
+    int32_t *rest = (int32_t *)malloc(n * sizeof(int32_t));
+    uint8_t *done = (uint8_t *)calloc(n, 1);
+    if (!A || !Wc || !S || !tcol || !rest || !done) {
+        free(A); free(Wc); free(S); free(tcol); free(rest); free(done);
+        return ORACLE_ERR_NOMEM;
+    }
+    memcpy(A, Hinv, n * n * sizeof(double));
+    for (size_t i = 0; i < m; ++i)
+        for (size_t j = 0; j < n; ++j) Wc[i * n + j] = (double)W[i * (size_t)ldw + j];
+
+    int status = ORACLE_OK;
+    size_t count = 0;
+    while (count < n && status == ORACLE_OK) {
+        /* scores of the remaining columns, from the current weights and the current diagonal */
+        size_t nrest = 0;
+        for (size_t j = 0; j < n; ++j) {
+            if (done[j]) continue;
+            double s = 0.0;
+            if (mode != SCORE_NONE) {
+                for (size_t i = 0; i < m; ++i) {
+                    const double w = Wc[i * n + j];
+                    double num;
+                    if (mode == SCORE_QERR || mode == SCORE_ERR) {
+                        const double sc = (double)scale[i], zp = (double)zero[i];
+                        const double q = dequant(quant_code(w, sc, zp, maxq), sc, zp);
+                        num = (w - q) * (w - q);
+                    } else {
+                        num = w * w;
+                    }
+                    if (mode == SCORE_QERR || mode == SCORE_PRUNE) s += num / (2.0 * A[j * n + j]);
+                    else s += num;
+                }
+            }
+            if (!isfinite(s)) { status = ORACLE_ERR_INVALID_ARG; break; }
+            S[j] = s;
+            rest[nrest++] = (int32_t)j;
+        }
+        if (status != ORACLE_OK) break;
+        g_sort_keys = S;
+        g_sort_ascending = ascending;
+        qsort(rest, nrest, sizeof(int32_t), cmp_score_stable);
+        const size_t take = nrest < (size_t)block ? nrest : (size_t)block;
+        for (size_t t = 0; t < take; ++t) {
+            const size_t p = (size_t)rest[t];
+            const double d = A[p * n + p];
+            if (!(d > 0.0) || !isfinite(d)) { status = ORACLE_ERR_NOT_SPD; break; }
+            const double *Ap = A + p * n;
+#pragma omp parallel for schedule(static)
+            for (size_t i = 0; i < m; ++i) {
+                double *w = Wc + i * n;
+                const double sc = (double)scale[i], zp = (double)zero[i];
+                if (prer) prer[i * n + p] = w[p] / sc;
+                const int c = quant_code(w[p], sc, zp, maxq);
+                const double q = dequant(c, sc, zp);
+                const double ei = (w[p] - q) / d;
+                for (size_t j = 0; j < n; ++j)
+                    if (!done[j] && j != p) w[j] -= ei * Ap[j]; /* Eq. 11 */
+                w[p] = q;
+                codes[i * n + p] = (uint8_t)c;
+            }
+            for (size_t j = 0; j < n; ++j) tcol[j] = A[j * n + p] / d;
+#pragma omp parallel for schedule(static)
+            for (size_t j = 0; j < n; ++j) { /* Eq. 12 on the columns still to come */
+                if (done[j] || j == p) continue;
+                double *Aj = A + j * n;
+                const double tj = tcol[j];
+                for (size_t k = 0; k < n; ++k)
+                    if (!done[k] && k != p) Aj[k] -= tj * Ap[k];
+            }
+            for (size_t j = 0; j < n; ++j) { A[p * n + j] = 0.0; A[j * n + p] = 0.0; }
+            done[p] = 1;
+            order_out[count++] = (int32_t)p;
+        }
+    }
+    if (status == ORACLE_OK) {
+        if (What)
+            for (size_t i = 0; i < m; ++i)
+                for (size_t j = 0; j < n; ++j) What[i * n + j] = (float)Wc[i * n + j];
+        if (H_undamped && loss_out) {
+            double total = 0.0;
+            for (size_t i = 0; i < m; ++i) {
+                double acc = 0.0;
+                for (size_t a = 0; a < n; ++a) {
+                    const double da = (double)W[i * (size_t)ldw + a] - (double)(float)Wc[i * n + a];
+                    double t = 0.0;
+                    for (size_t b = 0; b < n; ++b)
+                        t += H_undamped[a * n + b] * ((double)W[i * (size_t)ldw + b] - (double)(float)Wc[i * n + b]);
+                    acc += da * t;
+                }
+                total += 0.5 * acc;
+            }
+            *loss_out = total;
+        }
+    }
+    free(A); free(Wc); free(S); free(tcol); free(rest); free(done);
+    return status;
+}
+
+/* ---------------------------------------------------------------------------------------
+ * The non-parallel arm of the paper's ablation (Sec. 4.2, the paragraph on the per-row inverse
+ * Hessians; the rows of Table 3 without the parallel tick): every row is ranked and quantized on
+ * its own.  Row i sorts ITS weights by their own sensitivities L_ij (Sec. 4.1; the keys and tie
+ * rule of oracle_sensitivity_order applied to that single row) and runs the column loop in that
+ * order against a private copy of the inverse Hessian -- the [d_row, d_col, d_col] tensor, here
+ * one slice at a time.  Cost rows * cols^3 / 3: small layers only.
+ *   perm_rows [rows x cols]: the order each row used.
+ * ------------------------------------------------------------------------------------- */
+int oracle_quantize_layer_per_row(const float *W, int rows, int cols, int64_t ldw, const double *Hinv,
+                                  const double *Hinv_diag, const float *scale, const float *zero, int bits,
+                                  int mode_and_direction, uint8_t *codes, float *What, int32_t *perm_rows,
+                                  const double *H_undamped, double *loss_out) {
+    if (!W || !Hinv || !scale || !zero || !codes || !perm_rows || rows < 1 || cols < 1 || ldw < cols)
+        return ORACLE_ERR_INVALID_ARG;
+    const size_t n = (size_t)cols;
+    double *S = (double *)malloc(n * sizeof(double));
+    if (!S) return ORACLE_ERR_NOMEM;
+    double total = 0.0;
+    int status = ORACLE_OK;
+    for (int i = 0; i < rows && status == ORACLE_OK; ++i) {
+        const float *wi = W + (size_t)i * (size_t)ldw;
+        int32_t *perm = perm_rows + (size_t)i * n;
+        status = oracle_sensitivity_order(wi, 1, cols, ldw, Hinv_diag, scale + i, zero + i, bits,
+                                          mode_and_direction, S, perm);
+        if (status != ORACLE_OK) break;
+        double loss = 0.0;
+        status = oracle_quantize_layer_ex(wi, 1, cols, ldw, Hinv, perm, scale + i, zero + i, bits,
+                                          codes + (size_t)i * n, What ? What + (size_t)i * n : NULL, H_undamped,
+                                          H_undamped ? &loss : NULL, NULL, NULL, NULL, NULL, NULL);
+        total += loss;
+    }
+    if (status == ORACLE_OK && H_undamped && loss_out) *loss_out = total;
+    free(S);
+    return status;
 }

@@ -62,6 +62,16 @@ def test_scaling_shape_1024_square(bits):
     assert nm == 0
 
 
+@pytest.mark.parametrize("rows,cols,n", [(4096, 192, 512), (4800, 130, 400)])
+def test_tall_layers_reach_the_single_cta_and_wrapped_row_group_paths(rows, cols, n):
+    """Tall, narrow layers.  4096 rows are 128 row groups of 32, so every group of the sweep is served by one CTA that
+    owns all three column blocks; 4800 rows are 150 groups, more than the CTAs of the persistent sweep, so CTAs walk
+    several groups one after the other (and 130 columns leave a ragged last block).  Whole path, every weight."""
+    spec = wl.LayerSpec("tall", rows, cols, n, 4, "kaiming", "halfnormal", 900 + rows)
+    nm, _, _ = _full(spec)
+    assert nm == 0
+
+
 def _row_subset_parity(spec, sub_rows, seed):
     """Full GPU run; oracle Hessian / inverse / scores / order in full, oracle sweep on a seeded subset of rows."""
     W, X = wl.make_layer(spec)

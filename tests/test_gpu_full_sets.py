@@ -1,17 +1,12 @@
 """Parity of EVERY layer of the ResNet-50-shaped and YOLOv5s-shaped sets and of the scaling shapes against the CPU
-oracle.  The oracle needs several minutes for the sets, so these tests only run when PTQ_FULL_SETS=1 is set
-(`PTQ_FULL_SETS=1 python -m pytest tests/test_gpu_full_sets.py -m gpu -q`); the default GPU suite covers a
-representative subset of the same layers (tests/test_gpu_configs.py)."""
-import os
-
+oracle, layer by layer, at full size (a few minutes, nearly all of it oracle time on the host)."""
 import numpy as np
 import pytest
 
 from paper_2509_05576_b200 import workloads as wl
 from test_gpu_configs import _full, _row_subset_parity
 
-pytestmark = [pytest.mark.gpu,
-              pytest.mark.skipif(os.environ.get("PTQ_FULL_SETS") != "1", reason="set PTQ_FULL_SETS=1 to run")]
+pytestmark = pytest.mark.gpu
 
 _SETS = {"c3": wl.config3(), "c4w8": wl.config4(bits=(8,)), "c4w4": wl.config4(bits=(4,))}
 

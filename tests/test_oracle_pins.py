@@ -145,7 +145,14 @@ def test_grid_is_minmax_and_quant_is_nearest_level(bits):
         lo, hi = min(W[i].min(), 0.0), max(W[i].max(), 0.0)
         assert scale[i] == np.float32((float(hi) - float(lo)) / maxq)
         assert zero[i] == np.rint(zero[i]) and 0 <= zero[i] <= maxq
+        # the zero-point itself: level `zero` is the grid's 0, placed so that level 0 sits at the row minimum and the
+        # top level at the row maximum, each to within half a step (an off-by-one zero-point shifts the whole grid by
+        # one step and fails both)
+        assert zero[i] == np.rint(-float(lo) / ((float(hi) - float(lo)) / maxq))
         levels = float(scale[i]) * (np.arange(maxq + 1) - float(zero[i]))
+        half = 0.5 * float(scale[i]) * (1 + 1e-6)
+        assert abs(levels[0] - float(lo)) <= half and abs(levels[maxq] - float(hi)) <= half
+        assert levels[int(zero[i])] == 0.0
         for w in W[i].astype(np.float64):
             c = oracle.quant_code(w, scale[i], zero[i], bits)
             assert 0 <= c <= maxq
@@ -188,6 +195,16 @@ def test_ordering_hand_example():
     # diagonal inverse Hessian: no compensation, codes are round-to-nearest under either order
     out = oracle.quantize_layer(W, np.diag(g["hinv_diag"]), perm, scale, zero, bits)
     assert np.array_equal(out["codes"], np.stack([g["codes_row0"], g["codes_row1"]]).astype(np.uint8))
+    # ascending variants (Sec. 4.1): same scores, reversed order
+    for mode, key_s, key_o in [(oracle.SCORE_QERR, "s_qerr", "order_qerr_asc"),
+                               (oracle.SCORE_PRUNE, "s_prune", "order_prune_asc")]:
+        S, perm = oracle.sensitivity_order(W, g["hinv_diag"], scale, zero, bits, mode | oracle.SCORE_ASCENDING)
+        assert np.allclose(S, g[key_s], rtol=1e-6) and list(perm) == list(g[key_o].astype(int))
+    # the non-parallel arm: each row in its own order; codes are still round-to-nearest (diagonal inverse Hessian)
+    out = oracle.quantize_layer_per_row(W, np.diag(g["hinv_diag"]), g["hinv_diag"], scale, zero, bits)
+    assert list(out["perm_rows"][0]) == list(g["order_row0"].astype(int))
+    assert list(out["perm_rows"][1]) == list(g["order_row1"].astype(int))
+    assert np.array_equal(out["codes"], np.stack([g["codes_row0"], g["codes_row1"]]).astype(np.uint8))
 
 
 @pytest.mark.parametrize("mode", [oracle.SCORE_QERR, oracle.SCORE_PRUNE, oracle.SCORE_ERR, oracle.SCORE_W])
@@ -211,6 +228,28 @@ def test_scores_match_definition_and_sort_is_stable(mode):
     pos = {int(c): k for k, c in enumerate(perm)}
     assert S[3] == S[7] == S[15] and pos[3] < pos[7] < pos[15]
     assert pos[7] == pos[3] + 1 and pos[15] == pos[3] + 2
+
+
+@pytest.mark.parametrize("mode", [oracle.SCORE_QERR, oracle.SCORE_W])
+def test_ascending_order_is_stable_and_mirrors_descending(mode):
+    W, X = _small_layer(9, 24, 64, 22)
+    W[:, 7] = W[:, 3]
+    W[:, 15] = W[:, 3]
+    Hinv, diag, _ = oracle.prepare_hinv(oracle.hessian_accumulate(X))
+    diag[7] = diag[3]
+    diag[15] = diag[3]
+    scale, zero = oracle.minmax_grid(W, 3)
+    S_d, perm_d = oracle.sensitivity_order(W, diag, scale, zero, 3, mode)
+    S_a, perm_a = oracle.sensitivity_order(W, diag, scale, zero, 3, mode | oracle.SCORE_ASCENDING)
+    assert np.array_equal(S_a, S_d)                      # the direction changes the sort only
+    assert sorted(perm_a) == list(range(24)) and np.all(np.diff(S_a[perm_a]) >= 0)
+    pos = {int(c): k for k, c in enumerate(perm_a)}
+    assert pos[7] == pos[3] + 1 and pos[15] == pos[3] + 2        # ties: lower column index first, as descending
+    # away from the tie group the ascending order is the descending one read backwards
+    rest_a = [c for c in perm_a if c not in (3, 7, 15)]
+    rest_d = [c for c in perm_d if c not in (3, 7, 15)]
+    assert rest_a == rest_d[::-1]
+    assert list(perm_a) == list(np.argsort(S_a, kind="stable"))
 
 
 def test_score_none_is_identity_order():
@@ -297,6 +336,117 @@ def test_factor_form_identity():
     for p in range(14):
         Ap = A0 if p == 0 else out["A_trace"][p - 1]
         assert np.allclose(Ap[p, p:] / np.sqrt(Ap[p, p]), U[p, p:], rtol=1e-9, atol=1e-14)
+
+
+def test_oracle_factor_is_the_cholesky_factor_of_the_permuted_inverse():
+    W, X, H, Hinv, lam, scale, zero, perm, bits = _tiny(62, 4, 33, 80)
+    U = oracle.factor_upper(Hinv, perm)
+    A0 = Hinv[np.ix_(perm, perm)]
+    ref = np.linalg.cholesky(A0).T                       # LAPACK
+    assert np.all(np.tril(U, -1) == 0)
+    assert np.max(np.abs(U - ref)) <= 1e-12 * np.max(np.abs(ref))
+    assert np.max(np.abs(U.T @ U - A0)) <= 1e-13 * np.max(np.abs(A0))
+    with pytest.raises(oracle.OracleError) as ei:
+        oracle.factor_upper(-np.eye(3), np.arange(3, dtype=np.int32))
+    assert ei.value.code == oracle.ERR_NOT_SPD and ei.value.info == 0
+
+
+@pytest.mark.parametrize("rows,cols,n,bits,xdist", [(5, 9, 30, 3, "halfnormal"), (16, 64, 48, 4, "halfnormal"),
+                                                    (32, 130, 256, 4, "silu"), (24, 300, 200, 8, "normal"),
+                                                    (12, 1024, 1500, 4, "halfnormal_sparse30"),
+                                                    (8, 2304, 2048, 4, "halfnormal"), (6, 2304, 4096, 3, "halfnormal")])
+def test_factor_form_sweep_equals_the_literal_loop(rows, cols, n, bits, xdist):
+    """The factor-form mode against the literal Eq. 11 / Eq. 12 loop, up to the widest layers the literal loop
+    reaches (2304 columns, with fewer calibration columns than weight columns in one case): same codes, same What,
+    the same values before rounding."""
+    W, X = _small_layer(rows, cols, n, 300 + cols + bits, xdist)
+    H = oracle.hessian_accumulate(X)
+    Hinv, diag, lam = oracle.prepare_hinv(H)
+    scale, zero = oracle.minmax_grid(W, bits)
+    S, perm = oracle.sensitivity_order(W, diag, scale, zero, bits)
+    lit = oracle.quantize_layer(W, Hinv, perm, scale, zero, bits, want_prer=True)
+    U = oracle.factor_upper(Hinv, perm)
+    fac = oracle.quantize_rows_factor(W, U, perm, scale, zero, bits, want_prer=True)
+    assert np.max(np.abs(fac["prer"] - lit["prer"])) <= 1e-7
+    near = np.abs(np.abs(lit["prer"] - np.floor(lit["prer"])) - 0.5) <= 1e-6
+    differ = fac["codes"] != lit["codes"]
+    assert not np.any(differ & ~near)
+    if not differ.any():
+        assert np.array_equal(fac["What"], lit["What"])
+    # rows are independent in this mode too
+    sub = [rows - 1, 0]
+    part = oracle.quantize_rows_factor(W[sub], U, perm, scale[sub], zero[sub], bits)
+    assert np.array_equal(part["codes"], fac["codes"][sub])
+
+
+# ------------------------------------------------------------------ dynamic re-ranking (Sec. 5)
+@pytest.mark.parametrize("mode", [oracle.SCORE_QERR, oracle.SCORE_PRUNE | oracle.SCORE_ASCENDING])
+def test_dynamic_with_one_block_is_the_static_method(mode):
+    W, X, H, Hinv, lam, scale, zero, _, bits = _tiny(90, 7, 21, 64, bits=4)
+    diag = np.diag(Hinv).copy()
+    S, perm = oracle.sensitivity_order(W, diag, scale, zero, bits, mode)
+    ref = oracle.quantize_layer(W, Hinv, perm, scale, zero, bits, H_undamped=H, want_prer=True)
+    for block in (21, 1000):
+        dyn = oracle.quantize_layer_dynamic(W, Hinv, scale, zero, bits, block, mode, H_undamped=H, want_prer=True)
+        assert np.array_equal(dyn["order"], perm)
+        assert np.array_equal(dyn["codes"], ref["codes"]) and np.array_equal(dyn["What"], ref["What"])
+        assert np.array_equal(dyn["prer"], ref["prer"])
+        assert dyn["loss"] == pytest.approx(ref["loss"], rel=1e-12)
+
+
+@pytest.mark.parametrize("block", [1, 4])
+def test_dynamic_order_follows_its_definition(block):
+    """The state the dynamic loop ranks from is the state of the literal static loop run in the same column sequence:
+    replay that sequence with the static loop (traces on), recompute the scores of the remaining columns from the
+    traced weights and the traced inverse Hessian with numpy at every re-ranking point, and check that the dynamic
+    loop picked the top `block` of them, in order."""
+    bits = 3
+    W, X, H, Hinv, lam, scale, zero, _, _ = _tiny(91, 6, 13, 40, bits=bits)
+    n = 13
+    dyn = oracle.quantize_layer_dynamic(W, Hinv, scale, zero, bits, block, oracle.SCORE_QERR)
+    order = dyn["order"]
+    assert sorted(order) == list(range(n))
+    rep = oracle.quantize_layer(W, Hinv, order, scale, zero, bits, want_trace=True)
+    assert np.array_equal(rep["codes"], dyn["codes"]) and np.array_equal(rep["What"], dyn["What"])
+    sc, zp = scale.astype(np.float64)[:, None], zero.astype(np.float64)[:, None]
+    for k in range(0, n, block):
+        if k == 0:
+            Wcur, Acur = W.astype(np.float64)[:, order], Hinv[np.ix_(order, order)]
+        else:
+            Wcur, Acur = rep["W_trace"][k - 1], rep["A_trace"][k - 1]          # permuted by `order`
+        rem = np.arange(k, n)
+        w = Wcur[:, rem]
+        q = sc * (np.clip(np.rint(w / sc) + zp, 0, 2 ** bits - 1) - zp)
+        Srem = ((w - q) ** 2 / (2.0 * np.diag(Acur)[rem][None, :])).sum(axis=0)
+        # stable descending by score, ties by lower ORIGINAL column index
+        want = sorted(range(len(rem)), key=lambda t: (-Srem[t], order[rem[t]]))[:block]
+        assert [int(order[rem[t]]) for t in want] == [int(c) for c in order[k:k + block]]
+    # re-ranking changes the sequence on this layer (otherwise the test would not bite)
+    _, perm_static = oracle.sensitivity_order(W, np.diag(Hinv).copy(), scale, zero, bits)
+    assert not np.array_equal(order, perm_static)
+
+
+# ------------------------------------------------------------------ the non-parallel arm (Sec. 4.2)
+def test_per_row_mode_ranks_and_quantizes_every_row_on_its_own():
+    bits = 4
+    W, X, H, Hinv, lam, scale, zero, perm, _ = _tiny(92, 6, 17, 50, bits=bits)
+    diag = np.diag(Hinv).copy()
+    out = oracle.quantize_layer_per_row(W, Hinv, diag, scale, zero, bits, H_undamped=H)
+    Wd = W.astype(np.float64)
+    err2 = (Wd - _dequant(_rtn_codes(W, scale, zero, bits), scale, zero)) ** 2
+    L = err2 / (2.0 * diag[None, :])
+    total = 0.0
+    for i in range(6):
+        perm_i = np.argsort(-L[i], kind="stable").astype(np.int32)
+        assert np.array_equal(out["perm_rows"][i], perm_i)
+        one = oracle.quantize_layer(W[i:i + 1], Hinv, perm_i, scale[i:i + 1], zero[i:i + 1], bits, H_undamped=H)
+        assert np.array_equal(out["codes"][i], one["codes"][0]) and np.array_equal(out["What"][i], one["What"][0])
+        total += one["loss"]
+    assert out["loss"] == pytest.approx(total, rel=1e-12)
+    dW = Wd - out["What"].astype(np.float64)
+    assert out["loss"] == pytest.approx(0.5 * np.einsum("ij,jk,ik->", dW, H, dW), rel=1e-10)
+    # the rows do not share one order on this layer
+    assert any(not np.array_equal(out["perm_rows"][i], out["perm_rows"][0]) for i in range(1, 6))
 
 
 def test_loss_from_hessian_equals_loss_from_inputs():
