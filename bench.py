@@ -31,7 +31,7 @@ from paper_2509_05576_b200 import workloads as wl  # noqa: E402
 
 METRIC = "weights quantized per second, whole per-layer path (ms_per_step = layer quantize time)"
 UNIT = "weights/s"
-FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12      # 148 SMs x 64 FP64 FMA / clk x 1965 MHz = 37.2
+FP64_PEAK_BOUND_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12  # stated upper bound: 148 SMs x 64 FP64 FMA / clk x 1965 MHz = 37.2
 INT8_OVER_BF16 = 2.0                                   # nominal dense 4.5 / 2.25 PFLOP/s
 
 
@@ -201,6 +201,65 @@ def algorithmic_work(spec):
     }
 
 
+def measure_fp64_peak(ptq, torch, stream):
+    """Float64 throughput of this GPU, measured in this run with the library's probe kernels (eight independent
+    chains of FMAs, or of tensor-core m8n8k4 MMAs, per thread and nothing else): best of five launches of each kind,
+    timed with CUDA events on the launching stream after two warm-up launches."""
+    sink = torch.zeros(1, dtype=torch.float64, device="cuda")
+    out = {}
+    for kind, name, iters in ((0, "dfma", 100000), (1, "dmma", 20000)):
+        best = 0.0
+        for rep in range(7):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            flops = ptq.fp64_probe(kind, iters, sink, stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if rep >= 2:
+                best = max(best, flops / (a.elapsed_time(b) * 1e-3) / 1e12)
+        out[name + "_tflops"] = best
+    out["fp64_tflops"] = max(out["dfma_tflops"], out["dmma_tflops"])
+    out["bound_tflops"] = FP64_PEAK_BOUND_TFLOPS
+    out["how"] = ("ptq_fp64_probe: 4 CTAs x 256 threads per SM, 8 independent chains per thread, 100000 (FMA) / 20000 (MMA) "
+                  "rounds, best of 5 launches, CUDA events; bound = 148 SMs x 64 FMA/clk x 2 x 1.965 GHz")
+    return out
+
+
+def layer_set_totals(fp64_peak, flush, ws):
+    """The configurations beyond the single bench layer, measured in this run: the ResNet-50-shaped set (4-bit), the
+    YOLOv5s-shaped set (8- and 4-bit) and the scaling shapes at 3, 4 and 8 bits.  Per set: total ms, weights/s, per-stage
+    ms and per-stage roofline fraction (sum of algorithmic work / sum of stage time / peak)."""
+    from paper_2509_05576_b200 import layer_set_run as lsr
+
+    def brief(res, per_layer=False):
+        out = {k: res[k] for k in ("n_layers", "weights", "total_ms", "weights_per_s", "stage_total_ms",
+                                   "stage_roofline_frac")}
+        if per_layer:
+            out["layers"] = [{"layer": r["layer"], "ms": r["ms"], "stages_ms": r["stages_ms"],
+                              "roofline_frac": r["roofline_frac"]} for r in res["layers"]]
+        return out
+
+    sets = {}
+    sets["c3_resnet50_w4"] = brief(lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush))
+    # the YOLOv5s-shaped layers at 8 and 4 bits share their inputs: run the two bit-widths of a layer back to back
+    c4 = [s for pair in zip(wl.config4(bits=(8,)), wl.config4(bits=(4,))) for s in pair]
+    res4 = lsr.run_specs(c4, 2, fp64_peak=fp64_peak, ws=ws, flush=flush)
+    for b in (8, 4):
+        rows = [r for r in res4["layers"] if r["bits"] == b]
+        st = {}
+        for r in rows:
+            for k, v in r["stages_ms"].items():
+                st[k] = st.get(k, 0.0) + v
+        ms = sum(r["ms"] for r in rows)
+        wts = sum(r["rows"] * r["cols"] for r in rows)
+        sets[f"c4_yolov5s_w{b}"] = {"n_layers": len(rows), "weights": wts, "total_ms": ms,
+                                    "weights_per_s": wts / (ms * 1e-3), "stage_total_ms": st}
+    sets["c4_yolov5s_w8"]["stage_roofline_frac_both_bit_widths"] = res4["stage_roofline_frac"]
+    sets["c5_scaling_w3_w4_w8"] = brief(lsr.run_specs(wl.config5(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush),
+                                        per_layer=True)
+    return sets
+
+
 def kernel_rooflines(kernels, work, peaks):
     """Achieved rate of every kernel with a work model, against the peak of the unit that bounds it."""
     out = {}
@@ -213,8 +272,9 @@ def kernel_rooflines(kernels, work, peaks):
             peak, unit, ach = peaks["bf16_tflops"] * INT8_OVER_BF16, "TFLOP/s", per_s / 1e12
             note = f"int8 dense = {peaks['source']} bf16 burst {peaks['bf16_tflops']} TF/s x nominal ratio 2"
         elif bound == "alu":
-            peak, unit, ach = FP64_PEAK_TFLOPS, "TFLOP/s", per_s / 1e12
-            note = "float64 pipe: 148 SMs x 64 FMA/clk x 2 x 1965 MHz (a DFMA / DMMA microbenchmark reached 36.8)"
+            peak, unit, ach = peaks["fp64_tflops"], "TFLOP/s", per_s / 1e12
+            note = (f"float64 pipe, measured in this run by ptq_fp64_probe (FMA {peaks['fp64']['dfma_tflops']:.2f}, "
+                    f"MMA {peaks['fp64']['dmma_tflops']:.2f} TFLOP/s); stated upper bound {FP64_PEAK_BOUND_TFLOPS:.2f}")
         else:
             peak, unit, ach = peaks["hbm_gbs"], "GB/s", per_s / 1e9
             note = f"{peaks['source']} copy bandwidth"
@@ -302,6 +362,8 @@ def run_ours(args):
     kernels = {k: {"ms_per_step": ms / prof_steps, "launches_per_step": cnt // prof_steps} for k, (ms, cnt) in prof.items()}
     dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     peaks = load_peaks()
+    peaks["fp64"] = measure_fp64_peak(ptq, torch, stream)
+    peaks["fp64_tflops"] = peaks["fp64"]["fp64_tflops"]
     work = algorithmic_work(spec)
     per_kernel = kernel_rooflines(kernels, work, peaks)
     traffic = ncu_traffic(dominant)
@@ -314,8 +376,8 @@ def run_ours(args):
                     "launch_ms": dom["ms_per_step"] / dom_launches, "launches_per_step": dom["launches_per_step"],
                     "algorithmic_work_per_launch": work[dominant][1] / dom_launches}
     else:
-        roofline = {"kernel": dominant, "bound": "alu", "achieved": None, "peak": FP64_PEAK_TFLOPS, "unit": "TFLOP/s",
-                    "frac": None, "traffic": traffic}
+        roofline = {"kernel": dominant, "bound": "alu", "achieved": None, "peak": peaks["fp64_tflops"],
+                    "unit": "TFLOP/s", "frac": None, "traffic": traffic}
     roofline["per_kernel"] = per_kernel
     gram = per_kernel.get("gram_i8_tcgen05")
     if gram:
@@ -371,6 +433,12 @@ def run_ours(args):
                         "codes_equal_to_gpu": bool(np.array_equal(ref["codes"], bufs.codes.cpu().numpy())),
                         "order_equal_to_gpu": bool(np.array_equal(ref["perm"], bufs.perm.cpu().numpy()))}
 
+    # ---- the other configurations, measured in the same run (one GPU only)
+    layer_sets = None
+    if world == 1 and not args.no_sets:
+        del Wd, Xd
+        layer_sets = layer_set_totals(peaks["fp64_tflops"], flush, ws)
+
     if rank == 0:
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -378,7 +446,7 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": workload_config(spec, world), "clocks": clocks, "e2e": e2e,
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
-            "stages_ms": stage_ms, "kernels": kernels,
+            "stages_ms": stage_ms, "kernels": kernels, "fp64_peak": peaks["fp64"], "layer_sets": layer_sets,
             "context": "paper: ResNet-50 whole-model 80 s (FastOBQ) vs 9287 s (OBQ), hardware not stated"}))
     if world > 1:
         dist.destroy_process_group()
@@ -392,7 +460,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sets", action="store_true", help="skip the layer-set totals (the single bench layer only)")
     args = ap.parse_args()
+    if args.impl == "ours" and args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started plainly with --gpus N: become the launcher of N ranks, one per GPU
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(29500 + os.getpid() % 2000), os.path.abspath(__file__)]
+        return subprocess.call(cmd + sys.argv[1:])
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

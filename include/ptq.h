@@ -17,6 +17,10 @@
  *     before a sequence of calls and reads it after synchronising the stream.
  *   - Inputs are never modified; outputs are fully overwritten (H of ptq_hessian_accumulate is updated).
  *   - Results are deterministic: fixed reduction orders, no floating-point atomics.
+ *   - Host-side state (SM count, kernel attributes) is kept per device and looked up with the caller's current
+ *     device, so one process may drive several devices; calls may come from several host threads as long as calls
+ *     that share a stream, a workspace or output buffers are ordered by the caller.
+ *   - Size limits: ptq_quantize_layer takes rows <= 65535 and cols <= 65535 (PTQ_ERR_UNSUPPORTED beyond).
  *   - No exceptions, no exit(), no stdout, no device trap, no unbounded device-side wait.
  */
 #ifndef PTQ_H_
@@ -54,7 +58,11 @@ typedef enum {
     PTQ_SCORE_PRUNE = 1, /* Eq. 8 :  w^2 / (2 [Hinv]_jj) */
     PTQ_SCORE_ERR = 2,   /* (w - quant(w))^2 */
     PTQ_SCORE_W = 3,     /* w^2 */
-    PTQ_SCORE_NONE = 4   /* no sorting: identity order */
+    PTQ_SCORE_NONE = 4,  /* no sorting: identity order */
+    /* Sec. 4.1 names each key in a descending ("des") and an ascending ("asc") variant.  Descending is the default
+     * (and the method's); adding this flag to a mode sorts by S ascending.  Equal scores keep the lower column
+     * index first in both directions. */
+    PTQ_SCORE_ASCENDING = 16
 } ptq_score_mode;
 
 typedef enum {
@@ -119,8 +127,9 @@ int ptq_minmax_grid(const float *W, int rows, int cols, int64_t ldw, int bits, f
                     int32_t *status, void *stream);
 
 /*
- * Sec. 4.2 steps 1-3: S_j = sum_i score(w_ij) from the original W and diag(Hinv); perm = columns by S descending,
- * equal scores keep the lower column index first.   S [cols] float64 out, perm [cols] int32 out.
+ * Sec. 4.2 steps 1-3: S_j = sum_i score(w_ij) from the original W and diag(Hinv); perm = columns by S descending
+ * (ascending with PTQ_SCORE_ASCENDING added to score_mode), equal scores keep the lower column index first.
+ * S [cols] float64 out, perm [cols] int32 out.
  */
 int ptq_sensitivity_order(const float *W, int rows, int cols, int64_t ldw, const double *Hinv_diag, const float *scale,
                           const float *zero, int bits, int score_mode, double *S, int32_t *perm, void *ws,
@@ -140,9 +149,10 @@ int ptq_sensitivity_order(const float *W, int rows, int cols, int64_t ldw, const
  * Limits and rules
  *   - ceil(rows / 64) * cols * 8 bytes must not exceed PTQ_STATIC_SCRATCH_BYTES (e.g. 4096 x 11008 fits);
  *     larger problems return PTQ_ERR_STATIC_SCRATCH and launch nothing.
- *   - It never calls cudaMalloc, cudaFree or any allocating routine.  The first call on each device looks up the
- *     array's device address (cudaGetSymbolAddress, with the caller's device current) and keeps it; make that
- *     first call outside any stream capture.
+ *   - It never calls cudaMalloc, cudaFree or any allocating routine.  Every call looks up the array's device address
+ *     (cudaGetSymbolAddress, with the caller's device current; nothing is remembered between calls, so the address
+ *     is right after a cudaDeviceReset too).  The first such lookup on a device initialises the library's module
+ *     there: make the first call on each device outside any stream capture.
  *   - All calls on one device share the one array, and it keeps whatever the previous call left there.  The
  *     kernels overwrite every element they later read, so no clearing is needed; but two calls that may run at
  *     the same time on the GPU (different streams, or different host threads) race on it: keep calls to this
@@ -169,8 +179,35 @@ int ptq_quantize_layer(const float *W, int rows, int cols, int64_t ldw, const do
                        const double *H_undamped, double *loss_out, void *ws, size_t ws_bytes, int32_t *status,
                        void *stream);
 
+/*
+ * Sec. 4.2 step 3 alone: perm = the indices 0 .. cols-1 sorted by S descending (ascending != 0: ascending), equal
+ * scores keep the lower index first.  For callers that form S themselves, e.g. by summing the per-shard scores of a
+ * layer whose rows are spread over several GPUs (Sec. 4.2 step 2 is a sum over rows, so it splits over row shards).
+ *   S [cols] float64, perm [cols] int32 out.  No workspace.
+ */
+int ptq_sort_scores(const double *S, int cols, int ascending, int32_t *perm, void *stream);
+
 const char *ptq_status_string(int code);
 int ptq_version(void);
+
+/*
+ * Self-test of the bounded device-side waits (instrumentation; the paper has no counterpart).  Launches a kernel that
+ * calls the library's own wait routine on a target nothing will ever reach, with the given limit in SM clock cycles:
+ *   which = 0 : the grid-wide barrier of the factorisation kernel (one CTA per SM), asked for one arrival too many
+ *   which = 1 : the counter wait of the column sweep, on a counter that nobody raises
+ * The wait must run out, the kernel records {PTQ_ERR_TIMEOUT, CTA index, 1 + which} in `status` and returns; the
+ * context stays usable.  ws: at least 16 bytes of device scratch.  limit_cycles in [1, 4e9].
+ */
+int ptq_selftest_wait_timeout(int which, long long limit_cycles, void *ws, size_t ws_bytes, int32_t *status,
+                              void *stream);
+
+/*
+ * Float64 throughput probe (instrumentation; the paper has no counterpart): launches one kernel of 4 CTAs x 256 threads
+ * per SM in which every thread runs `iters` rounds of eight independent chains of float64 FMAs (kind 0) or of float64
+ * tensor-core MMAs m8n8k4 (kind 1), and nothing else.  *flops_out (host) receives the floating-point operations of
+ * that launch (FMA = 2); the caller times the launch on its stream.  sink: one device double (never written).
+ */
+int ptq_fp64_probe(int kind, int iters, double *sink, double *flops_out, void *stream);
 
 /*
  * Launch accounting (instrumentation; the paper has no counterpart).  Host-side state of the calling process.

@@ -6,8 +6,6 @@
 #include "colloop.cuh"
 #include "gram.cuh"
 
-#include <mutex>
-
 using namespace ptq;
 
 namespace {
@@ -25,6 +23,7 @@ inline int grid_x_for(int n, int threads) {
 }
 
 // The loss product is cut along k into as many slices as it takes to put about two CTAs on every SM.
+constexpr int kMaxGridY = 65535;
 constexpr int kLossMaxSplit = 8;
 int loss_ksplit(int rows, int cols) {
     const long ctas = (long)cdiv(rows, 64) * ((cdiv(cols, 64) + 1) / 2);
@@ -40,24 +39,86 @@ constexpr size_t kStaticScratchDoubles = PTQ_STATIC_SCRATCH_BYTES / sizeof(doubl
 static __device__ __align__(256) double g_static_score_scratch[kStaticScratchDoubles];
 
 // Device address of the array on the current device.  In host code the symbol's name is only a handle, so the
-// address is asked for once per device (with that device current) and remembered.
+// address is asked of the runtime, with the caller's device current, on every call: the lookup is cheap after the
+// first one, and an address remembered across a cudaDeviceReset or under another context would be stale.
 int static_scratch_address(double** out) {
-    constexpr int kMaxDevices = 64;
-    static std::mutex mu;
-    static double* addr[kMaxDevices] = {};
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PTQ_ERR_CUDA;
-    std::lock_guard<std::mutex> lock(mu);
-    if (!addr[dev]) {
-        double* p = nullptr;
-        if (cudaGetSymbolAddress((void**)&p, g_static_score_scratch) != cudaSuccess || !p) {
-            cudaGetLastError();
-            return PTQ_ERR_CUDA;
-        }
-        addr[dev] = p;
+    double* p = nullptr;
+    if (cudaGetSymbolAddress((void**)&p, g_static_score_scratch) != cudaSuccess || !p) {
+        cudaGetLastError();
+        return PTQ_ERR_CUDA;
     }
-    *out = addr[dev];
+    *out = p;
     return PTQ_OK;
+}
+
+// Scores and order (Sec. 4.2 steps 1-3) with the per-row-chunk partial sums in `partial`.
+int order_launch(const float* W, int rows, int cols, int64_t ldw, const double* Hinv_diag, const float* scale,
+                 const float* zero, int bits, int mode, int ascending, double* S, int32_t* perm, double* partial,
+                 int32_t* status, cudaStream_t stream) {
+    const int chunks = cdiv(rows, kScoreRowChunk);
+    if (chunks > 65535) return PTQ_ERR_UNSUPPORTED;
+    if (mode != PTQ_SCORE_NONE) {
+        Launch l(K_SCORE_PARTIAL, stream);
+        score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
+                                                                              mode, partial);
+    }
+    { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, mode, S, status); }
+    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, ascending, perm); }
+    return launch_status();
+}
+
+int order_args_check(const float* W, int rows, int cols, int64_t ldw, const double* Hinv_diag, const float* scale,
+                     const float* zero, int bits, int score_mode, const double* S, const int32_t* perm) {
+    if (!W || !S || !perm || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8) return PTQ_ERR_INVALID_ARG;
+    if (score_mode & ~(PTQ_SCORE_ASCENDING | 7)) return PTQ_ERR_INVALID_ARG;
+    const int mode = score_mode & ~PTQ_SCORE_ASCENDING;
+    if (mode < PTQ_SCORE_QERR || mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
+    if ((mode == PTQ_SCORE_QERR || mode == PTQ_SCORE_PRUNE) && !Hinv_diag) return PTQ_ERR_INVALID_ARG;
+    if ((mode == PTQ_SCORE_QERR || mode == PTQ_SCORE_ERR) && (!scale || !zero)) return PTQ_ERR_INVALID_ARG;
+    return PTQ_OK;
+}
+
+// Self-test kernels: they call the very wait routines of the factorisation and of the sweep on a target that nothing
+// will ever reach, so that the wait must run out, report PTQ_ERR_TIMEOUT and return.
+__global__ void __launch_bounds__(kCholThreads) selftest_barrier_kernel(unsigned* bar, int32_t* status, long long spin_limit) {
+    __shared__ int s_flag;
+    const bool ok = grid_barrier(bar, gridDim.x + 1u, &s_flag, spin_limit);      // one arrival more than the grid has
+    if (!ok && threadIdx.x == 0) report(status, PTQ_ERR_TIMEOUT, blockIdx.x, 1);
+}
+__global__ void selftest_counter_kernel(unsigned* words, int32_t* status, long long spin_limit) {
+    if (threadIdx.x == 0 && !bounded_counter_wait(&words[0], 1u, &words[1], spin_limit))
+        report(status, PTQ_ERR_TIMEOUT, blockIdx.x, 2);
+}
+
+// Float64 throughput probes: eight independent chains per thread, nothing but the arithmetic instruction in the loop.
+constexpr int kProbeThreads = 256, kProbeCtasPerSm = 4, kProbeChains = 8;
+__global__ void __launch_bounds__(kProbeThreads) fp64_probe_fma_kernel(int iters, double* sink) {
+    double acc[kProbeChains];
+    const double a = 1.0 + 1e-9 * threadIdx.x, b = 1e-12 * (blockIdx.x + 1);
+#pragma unroll
+    for (int c = 0; c < kProbeChains; ++c) acc[c] = (double)c;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int c = 0; c < kProbeChains; ++c) acc[c] = fma(acc[c], a, b);
+    }
+    double s = 0.0;
+#pragma unroll
+    for (int c = 0; c < kProbeChains; ++c) s += acc[c];
+    if (s == 123.456) sink[0] = s;          // never true: keeps the loop alive without a store per thread
+}
+__global__ void __launch_bounds__(kProbeThreads) fp64_probe_mma_kernel(int iters, double* sink) {
+    double acc[kProbeChains][2];
+    const double a = 1.0 + 1e-9 * threadIdx.x, b = 1e-3 * ((threadIdx.x & 3) + 1);
+#pragma unroll
+    for (int c = 0; c < kProbeChains; ++c) acc[c][0] = acc[c][1] = 1e-12 * c;
+    for (int it = 0; it < iters; ++it) {
+#pragma unroll
+        for (int c = 0; c < kProbeChains; ++c) dmma_884(acc[c][0], acc[c][1], a, b);
+    }
+    double s = 0.0;
+#pragma unroll
+    for (int c = 0; c < kProbeChains; ++c) s += acc[c][0] + acc[c][1];
+    if (s == 123.456) sink[0] = s;
 }
 
 }  // namespace
@@ -166,6 +227,7 @@ int ptq_hessian_accumulate_f64(double* H, const float* X, int cols, int n, int64
     (void)status;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!H || !X || cols < 1 || n < 1 || ldx < n) return PTQ_ERR_INVALID_ARG;
+    if (cols > kMaxGridY) return PTQ_ERR_UNSUPPORTED;
     if (!aligned16(H) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_HESSIAN_ACCUMULATE_F64, 0, cols, n)) return PTQ_ERR_WORKSPACE;
     Carver cv(ws);
@@ -249,47 +311,83 @@ int ptq_sensitivity_order(const float* W, int rows, int cols, int64_t ldw, const
                           const float* zero, int bits, int score_mode, double* S, int32_t* perm, void* ws,
                           size_t ws_bytes, int32_t* status, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    if (!W || !S || !perm || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8) return PTQ_ERR_INVALID_ARG;
-    if (score_mode < PTQ_SCORE_QERR || score_mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
-    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_PRUNE) && !Hinv_diag) return PTQ_ERR_INVALID_ARG;
-    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_ERR) && (!scale || !zero)) return PTQ_ERR_INVALID_ARG;
+    const int bad = order_args_check(W, rows, cols, ldw, Hinv_diag, scale, zero, bits, score_mode, S, perm);
+    if (bad) return bad;
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_SENSITIVITY_ORDER, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
     if (!aligned16(ws)) return PTQ_ERR_ALIGNMENT;
     Carver cv(ws);
-    const int chunks = cdiv(rows, kScoreRowChunk);
-    double* partial = cv.take<double>((size_t)chunks * cols);
-    if (score_mode != PTQ_SCORE_NONE) {
-        Launch l(K_SCORE_PARTIAL, stream);
-        score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
-                                                                              score_mode, partial);
-    }
-    { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status); }
-    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, perm); }
-    return launch_status();
+    double* partial = cv.take<double>((size_t)cdiv(rows, kScoreRowChunk) * cols);
+    return order_launch(W, rows, cols, ldw, Hinv_diag, scale, zero, bits, score_mode & ~PTQ_SCORE_ASCENDING,
+                        (score_mode & PTQ_SCORE_ASCENDING) ? 1 : 0, S, perm, partial, status, stream);
 }
 
 int ptq_sensitivity_order_static(const float* W, int rows, int cols, int64_t ldw, const double* Hinv_diag,
                                  const float* scale, const float* zero, int bits, int score_mode, double* S,
                                  int32_t* perm, int32_t* status, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    if (!W || !S || !perm || rows < 1 || cols < 1 || ldw < cols || bits < 2 || bits > 8) return PTQ_ERR_INVALID_ARG;
-    if (score_mode < PTQ_SCORE_QERR || score_mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
-    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_PRUNE) && !Hinv_diag) return PTQ_ERR_INVALID_ARG;
-    if ((score_mode == PTQ_SCORE_QERR || score_mode == PTQ_SCORE_ERR) && (!scale || !zero)) return PTQ_ERR_INVALID_ARG;
-    const int chunks = cdiv(rows, kScoreRowChunk);
-    if ((size_t)chunks * (size_t)cols > kStaticScratchDoubles) return PTQ_ERR_STATIC_SCRATCH;
+    const int bad = order_args_check(W, rows, cols, ldw, Hinv_diag, scale, zero, bits, score_mode, S, perm);
+    if (bad) return bad;
+    if ((size_t)cdiv(rows, kScoreRowChunk) * (size_t)cols > kStaticScratchDoubles) return PTQ_ERR_STATIC_SCRATCH;
     double* partial = nullptr;
     const int st = static_scratch_address(&partial);
     if (st) return st;
     // Every partial[ch][j] that score_final_kernel reads is written first by score_partial_kernel, so nothing
     // left in the array by an earlier call is ever used and nothing needs clearing.
-    if (score_mode != PTQ_SCORE_NONE) {
-        Launch l(K_SCORE_PARTIAL, stream);
-        score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
-                                                                              score_mode, partial);
+    return order_launch(W, rows, cols, ldw, Hinv_diag, scale, zero, bits, score_mode & ~PTQ_SCORE_ASCENDING,
+                        (score_mode & PTQ_SCORE_ASCENDING) ? 1 : 0, S, perm, partial, status, stream);
+}
+
+int ptq_sort_scores(const double* S, int cols, int ascending, int32_t* perm, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!S || !perm || cols < 1) return PTQ_ERR_INVALID_ARG;
+    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, ascending ? 1 : 0, perm); }
+    return launch_status();
+}
+
+int ptq_selftest_wait_timeout(int which, long long limit_cycles, void* ws, size_t ws_bytes, int32_t* status,
+                              void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if ((which != 0 && which != 1) || limit_cycles < 1 || limit_cycles > kSpinLimitCycles || !status)
+        return PTQ_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < 4 * sizeof(unsigned)) return PTQ_ERR_WORKSPACE;
+    if (!aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    unsigned* words = static_cast<unsigned*>(ws);
+    if (cudaMemsetAsync(words, 0, 4 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
+    if (which == 1) {
+        Launch l(K_SELFTEST, stream);
+        selftest_counter_kernel<<<1, 32, 0, stream>>>(words, status, limit_cycles);
+        return launch_status();
     }
-    { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, score_mode, S, status); }
-    { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, perm); }
+    DeviceState* dev = nullptr;
+    const int st = current_device_state(&dev);
+    if (st) return st;
+    if (!dev->coop) return PTQ_ERR_UNSUPPORTED;
+    void* args[] = {&words, &status, &limit_cycles};
+    Launch l(K_SELFTEST, stream);
+    if (cudaLaunchCooperativeKernel((const void*)selftest_barrier_kernel, dim3(dev->sms), dim3(kCholThreads), args, 0,
+                                    stream) != cudaSuccess) {
+        cudaGetLastError();
+        return PTQ_ERR_CUDA;
+    }
+    return PTQ_OK;
+}
+
+int ptq_fp64_probe(int kind, int iters, double* sink, double* flops_out, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if ((kind != 0 && kind != 1) || iters < 1 || iters > (1 << 24) || !sink || !flops_out) return PTQ_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    const int st = current_device_state(&dev);
+    if (st) return st;
+    const int grid = dev->sms * kProbeCtasPerSm;
+    const double threads = (double)grid * kProbeThreads;
+    Launch l(K_FP64_PROBE, stream);
+    if (kind == 0) {
+        fp64_probe_fma_kernel<<<grid, kProbeThreads, 0, stream>>>(iters, sink);
+        *flops_out = threads * kProbeChains * (double)iters * 2.0;
+    } else {
+        fp64_probe_mma_kernel<<<grid, kProbeThreads, 0, stream>>>(iters, sink);
+        *flops_out = (threads / 32.0) * kProbeChains * (double)iters * (8.0 * 8.0 * 4.0 * 2.0);
+    }
     return launch_status();
 }
 
@@ -301,6 +399,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     if (!W || !Hinv || !perm || !scale || !zero || !codes || rows < 1 || cols < 1 || ldw < cols || bits < 2 ||
         bits > 8)
         return PTQ_ERR_INVALID_ARG;
+    if (rows > kMaxGridY || cols > kMaxGridY) return PTQ_ERR_UNSUPPORTED;     // rows / columns index the grid's y dimension
     if (!aligned16(Hinv) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
     const int n = cols;

@@ -68,7 +68,8 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 }
 
 // bar[0]: arrival counter (monotonic, zero at launch), bar[1]: abort word.  Returns false when the CTA must leave.
-__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int* s_flag) {
+// spin_limit: SM clock cycles after which the wait gives up.
+__device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int* s_flag, long long spin_limit) {
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -79,7 +80,7 @@ __device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int
         while (ld_acquire_u32(&bar[0]) < target) {
             if ((++it & 63u) == 0u) {
                 if (ld_acquire_u32(&bar[1]) != 0u) { ok = 0; break; }
-                if (clock64() - t0 > 4000000000LL) { atomicExch(&bar[1], 1u); ok = 0; break; }
+                if (clock64() - t0 > spin_limit) { atomicExch(&bar[1], 1u); ok = 0; break; }
             }
         }
         __threadfence();
@@ -457,7 +458,7 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int6
 
 __global__ void __launch_bounds__(kCholThreads, 1)
 chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __restrict__ Dbuf, int n, int64_t ld,
-                 int vec16, unsigned* bar, int32_t* status) {
+                 int vec16, unsigned* bar, int32_t* status, long long spin_limit) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
     int* s_flag = reinterpret_cast<int*>(opnd + 2 * 2 * kNB * kCholLd);     // the strip panels alias opnd
@@ -571,7 +572,7 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
     strip_phase(0);
     for (int k = 0; k + 1 < nb; ++k) {
         ++epoch;
-        if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
+        if (!grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) break;
         // Block row k is final; the updates of block rows < k have been applied everywhere.
         const int next_items = strip_items(k + 1) > 0 ? strip_items(k + 1) : 1;
         // Look-ahead pays when giving up next_items CTAs lengthens the trailing phase by less than the strip phase and
@@ -607,14 +608,14 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         } else {
             trailing_phase(k, k + 1, 0);
             ++epoch;
-            if (!grid_barrier(bar, epoch * (unsigned)G, s_flag)) break;
+            if (!grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) break;
             strip_phase(k + 1);
         }
     }
     cp_async_wait<0>();
     // the diagonal factors move from the side buffer into A once nobody reads the original diagonal blocks any more
     ++epoch;
-    if (grid_barrier(bar, epoch * (unsigned)G, s_flag)) {
+    if (grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) {
         for (int b = blockIdx.x; b < nb; b += G)
             for (int idx = tid; idx < kNB * kNB; idx += kCholThreads) {
                 const int r = idx >> 6, c = idx & 63;
@@ -627,30 +628,31 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
 
 // In-place blocked upper Cholesky A = U^T U of the n x n matrix A (row stride n).  Only the upper triangle is read or
 // written.  With Wm (n x n, zero on entry) the same sweep also leaves W = U^-T there (lower triangular): the row
-// operations of the factorisation are applied to the identity, Sec. 5 item 1's "inverse of the decomposed result".
+// operations of the factorisation are applied to the identity, which gives the inverse of the Cholesky factor that
+// Sec. 5 item 1 asks for.
 // `bar` is 2 x uint32 of device scratch, Dbuf holds chol_scratch_doubles(n) doubles (the diagonal factors on their way).
 inline size_t chol_scratch_doubles(int n) { return (size_t)((n + kNB - 1) / kNB) * kNB * kNB; }
 inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* bar, int32_t* status,
                           cudaStream_t stream) {
-    static int grid = 0;
-    if (grid == 0) {
-        if (cudaFuncSetAttribute(chol_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kCholSmemBytes) != cudaSuccess)
-            return PTQ_ERR_CUDA;
-        int dev = 0, sms = 0, per_sm = 0, coop = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-        if (!coop) return PTQ_ERR_UNSUPPORTED;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chol_coop_kernel, kCholThreads, kCholSmemBytes) !=
-                cudaSuccess || per_sm < 1)
-            return PTQ_ERR_CUDA;
-        grid = sms;          // one CTA per SM: the cooperative launch guarantees that all of them are resident
-    }
+    DeviceState* dev = nullptr;
+    int st = current_device_state(&dev);
+    if (st) return st;
+    if (!dev->coop) return PTQ_ERR_UNSUPPORTED;
+    st = ensure_smem_attr(dev, SA_CHOL, [] {
+        cudaError_t e = cudaFuncSetAttribute(chol_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kCholSmemBytes);
+        int per_sm = 0;
+        if (e == cudaSuccess)
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, chol_coop_kernel, kCholThreads, kCholSmemBytes);
+        return (e == cudaSuccess && per_sm < 1) ? cudaErrorLaunchOutOfResources : e;
+    });
+    if (st) return st;
+    const int grid = dev->sms;   // one CTA per SM: the cooperative launch guarantees that all of them are resident
     if (cudaMemsetAsync(bar, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int64_t ld = n;
     int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;
-    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status};
+    long long spin_limit = kSpinLimitCycles;
+    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status, &spin_limit};
     Launch l(K_CHOL_COOP, stream);
     if (cudaLaunchCooperativeKernel((const void*)chol_coop_kernel, dim3(grid), dim3(kCholThreads), args,
                                     kCholSmemBytes, stream) != cudaSuccess) {

@@ -86,7 +86,23 @@ struct SweepParams {
     int rows, n, bits, vec16;
     unsigned* flags;        // [groups] published 8-column pieces of E per group, then [1] abort word; zero at launch
     int32_t* status;
+    long long spin_limit;   // SM clock cycles after which a wait on another CTA gives up
 };
+
+// Waits (one thread) until *counter >= target.  Gives up when the abort word is raised or after spin_limit cycles, in
+// which case it raises the abort word itself.  Returns whether the target was reached.
+__device__ __forceinline__ bool bounded_counter_wait(const unsigned* counter, unsigned target, unsigned* abort_word,
+                                                     long long spin_limit) {
+    const long long t0 = clock64();
+    unsigned it = 0;
+    while (ld_acquire_u32(counter) < target) {
+        if ((++it & 63u) == 0u) {
+            if (ld_acquire_u32(abort_word) != 0u) return false;
+            if (clock64() - t0 > spin_limit) { atomicExch(abort_word, 1u); return false; }
+        }
+    }
+    return true;
+}
 
 // Copies a tile of nr x nc doubles (nc even when vec16) from src (row stride ld) into dst (row stride dst_ld);
 // rows at or beyond rmax and columns at or beyond cmax are filled with zeros.
@@ -314,7 +330,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                                 if (m > 0) {
                                     const long long t0 = clock64();
                                     while (*s_pub != 8 * b + m) {
-                                        if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); break; }
+                                        if (clock64() - t0 > prm.spin_limit) { atomicExch(abort_word, 1u); break; }
                                     }
                                 }
                                 // a reduction without a return value: the warp does not wait for the round trip, and
@@ -346,15 +362,8 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
             } else if (!next_mine && !next2_mine) {
                 // ------------------------------------------------------------ wait for all of E[:, b]
                 if (tid == 0) {
-                    const long long t0 = clock64();
-                    int ok = 1;
-                    unsigned it = 0;
-                    while (ld_acquire_u32(&prm.flags[g]) < (unsigned)(8 * (b + 1))) {
-                        if ((++it & 63u) == 0u) {
-                            if (ld_acquire_u32(abort_word) != 0u) { ok = 0; break; }
-                            if (clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); ok = 0; break; }
-                        }
-                    }
+                    const int ok = bounded_counter_wait(&prm.flags[g], (unsigned)(8 * (b + 1)), abort_word,
+                                                        prm.spin_limit) ? 1 : 0;
                     __threadfence();
                     *s_flag = ok;
                 }
@@ -425,7 +434,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                             if (__all_sync(0xffffffffu, have)) break;
                             if ((++it & 15u) == 0u) {
                                 bool bad = ld_acquire_u32(abort_word) != 0u;
-                                if (!bad && clock64() - t0 > 4000000000LL) { atomicExch(abort_word, 1u); bad = true; }
+                                if (!bad && clock64() - t0 > prm.spin_limit) { atomicExch(abort_word, 1u); bad = true; }
                                 if (__any_sync(0xffffffffu, bad)) { ok = false; break; }
                             }
                         }
@@ -537,21 +546,20 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 // Launches the sweep: one CTA per SM, cooperative so that every CTA a waiting CTA depends on is resident.
 inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p, const float* scale, const float* zero,
                         int rows, int n, int bits, unsigned* flags, int32_t* status, cudaStream_t stream) {
-    static int grid = 0;
-    if (grid == 0) {
-        if (cudaFuncSetAttribute(sweep_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kSweepSmemBytes) != cudaSuccess)
-            return PTQ_ERR_CUDA;
-        int dev = 0, sms = 0, per_sm = 0, coop = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-        if (!coop) return PTQ_ERR_UNSUPPORTED;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_coop_kernel, kSweepThreads,
-                                                          kSweepSmemBytes) != cudaSuccess || per_sm < 1)
-            return PTQ_ERR_CUDA;
-        grid = sms;
-    }
+    DeviceState* dev = nullptr;
+    int st = current_device_state(&dev);
+    if (st) return st;
+    if (!dev->coop) return PTQ_ERR_UNSUPPORTED;
+    st = ensure_smem_attr(dev, SA_SWEEP, [] {
+        cudaError_t e = cudaFuncSetAttribute(sweep_coop_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kSweepSmemBytes);
+        int per_sm = 0;
+        if (e == cudaSuccess)
+            e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, sweep_coop_kernel, kSweepThreads, kSweepSmemBytes);
+        return (e == cudaSuccess && per_sm < 1) ? cudaErrorLaunchOutOfResources : e;
+    });
+    if (st) return st;
+    const int grid = dev->sms;
     const int groups = cdiv(rows, kSweepRows);
     if (cudaMemsetAsync(flags, 0, ((size_t)groups + 1) * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     // every byte 0xFF is a NaN: "not published yet" for the owner of the next block, which polls the values themselves
@@ -560,7 +568,7 @@ inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p
     prm.Wp = Wp; prm.U = U; prm.E = E; prm.codes_p = codes_p; prm.scale = scale; prm.zero = zero;
     prm.rows = rows; prm.n = n; prm.bits = bits;
     prm.vec16 = ((n & 1) == 0 && aligned16(Wp) && aligned16(U) && aligned16(E)) ? 1 : 0;
-    prm.flags = flags; prm.status = status;
+    prm.flags = flags; prm.status = status; prm.spin_limit = kSpinLimitCycles;
     void* args[] = {&prm};
     Launch l(K_SWEEP_COOP, stream);
     if (cudaLaunchCooperativeKernel((const void*)sweep_coop_kernel, dim3(grid), dim3(kSweepThreads), args,

@@ -4,6 +4,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 #include <stddef.h>
+#include <mutex>
 #include <vector>
 
 #include "../../include/ptq.h"
@@ -82,6 +83,49 @@ inline int launch_status() { return cudaGetLastError() == cudaSuccess ? PTQ_OK :
 
 inline int cdiv(int a, int b) { return (a + b - 1) / b; }
 
+// Bounded device-side waits give up after this many SM clock cycles (about two seconds).
+constexpr long long kSpinLimitCycles = 4000000000LL;
+
+// ---------------------------------------------------------------------------------------------------------
+// Host-side state that belongs to a DEVICE, not to the process: the SM count that sizes the persistent grids, the
+// cooperative-launch capability and which kernels already carry their dynamic shared-memory attribute there
+// (cudaFuncSetAttribute is per device).  One table, one mutex; looked up with the caller's device current.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kMaxDevices = 64;
+enum SmemAttrSlot { SA_CHOL = 0, SA_SWEEP, SA_GRAM, SA_DGEMM, SA_SMALL, SA_PROBE, SA_COUNT };
+struct DeviceState {
+    int sms = 0;
+    int coop = 0;
+    bool attr[SA_COUNT] = {};
+};
+inline std::mutex& host_state_mutex() { static std::mutex mu; return mu; }
+inline int current_device_state(DeviceState** out) {
+    static DeviceState table[kMaxDevices];
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return PTQ_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(host_state_mutex());
+    DeviceState& d = table[dev];
+    if (d.sms == 0) {
+        int sms = 0, coop = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return PTQ_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess) return PTQ_ERR_CUDA;
+        d.coop = coop;
+        d.sms = sms;
+    }
+    *out = &d;
+    return PTQ_OK;
+}
+// Runs `set` (the cudaFuncSetAttribute calls of one kernel family) once per device.
+template <typename F>
+inline int ensure_smem_attr(DeviceState* d, SmemAttrSlot slot, F set) {
+    std::lock_guard<std::mutex> lock(host_state_mutex());
+    if (!d->attr[slot]) {
+        if (set() != cudaSuccess) { cudaGetLastError(); return PTQ_ERR_CUDA; }
+        d->attr[slot] = true;
+    }
+    return PTQ_OK;
+}
+
 // ---------------------------------------------------------------------------------------------------------
 // Launch accounting.  Every kernel launch of the library goes through a Launch scope: it always counts the
 // launch, and, while profiling is enabled, brackets it with CUDA events on the launching stream so that the
@@ -92,7 +136,7 @@ enum KernelId {
     K_GRAM_SPLIT = 0, K_GRAM_I8, K_GRAM_FINISH, K_CONVERT_F64, K_DGEMM_GRAM, K_LAMBDA, K_DAMP_COPY, K_CHOL_COOP,
     K_DGEMM_LAUUM, K_EXTRACT_DIAG, K_MINMAX_GRID, K_SCORE_PARTIAL,
     K_SCORE_FINAL, K_RANK_SORT, K_PERM_CHECK, K_GATHER_SYM, K_GATHER_W, K_SWEEP_COOP, K_FINALIZE,
-    K_DGEMM_LOSS, K_SUM_PARTIALS, K_COUNT
+    K_DGEMM_LOSS, K_SUM_PARTIALS, K_SELFTEST, K_FP64_PROBE, K_COUNT
 };
 
 inline const char* kernel_name(int id) {
@@ -100,7 +144,7 @@ inline const char* kernel_name(int id) {
         "gram_split", "gram_i8_tcgen05", "gram_finish", "convert_f64", "dgemm_gram_f64", "lambda", "damp_copy", "chol_coop",
         "dgemm_lauum", "extract_diag",
         "minmax_grid", "score_partial", "score_final", "rank_sort", "perm_check", "gather_sym", "gather_w",
-        "sweep_coop", "finalize", "dgemm_loss", "sum_partials"};
+        "sweep_coop", "finalize", "dgemm_loss", "sum_partials", "selftest_wait", "fp64_probe"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 
@@ -123,15 +167,22 @@ struct Profiler {
 };
 inline Profiler& profiler() { static Profiler p; return p; }
 
+inline std::mutex& profiler_mutex() { static std::mutex mu; return mu; }
+
 struct Launch {
     int id; cudaStream_t s; cudaEvent_t a = nullptr, b = nullptr;
     Launch(int id_, cudaStream_t s_) : id(id_), s(s_) {
+        std::lock_guard<std::mutex> lock(profiler_mutex());
         Profiler& p = profiler();
         ++p.launches[id];
         if (p.on) { a = p.get(); b = p.get(); if (a) cudaEventRecord(a, s); }
     }
     ~Launch() {
-        if (a && b) { cudaEventRecord(b, s); profiler().recs.push_back({id, a, b}); }
+        if (a && b) {
+            cudaEventRecord(b, s);
+            std::lock_guard<std::mutex> lock(profiler_mutex());
+            profiler().recs.push_back({id, a, b});
+        }
     }
 };
 

@@ -291,19 +291,23 @@ inline GemmParams gemm_defaults() {
 // Launches with 128x128 tiles when that still fills the GPU, else 64x64.  Also reports the grid used.
 inline int launch_dgemm(int kernel_id, const GemmParams& p, int batches, cudaStream_t stream, int force_bt = 0,
                         dim3* grid_out = nullptr) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaFuncSetAttribute(dgemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)gemm_smem_bytes<128>());
-        cudaFuncSetAttribute(dgemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)gemm_smem_bytes<64>());
-        attr_done = true;
-    }
+    DeviceState* dev = nullptr;
+    int dst = current_device_state(&dev);
+    if (dst) return dst;
+    dst = ensure_smem_attr(dev, SA_DGEMM, [] {
+        cudaError_t e = cudaFuncSetAttribute(dgemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)gemm_smem_bytes<128>());
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(dgemm_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)gemm_smem_bytes<64>());
+        return e;
+    });
+    if (dst) return dst;
     if (p.M <= 0 || p.N <= 0 || batches <= 0) return PTQ_OK;
     int bt = force_bt;
     if (bt == 0) {
         const long tiles128 = (long)cdiv(p.M, 128) * cdiv(p.N, 128) * batches / (p.upper_only ? 2 : 1);
-        bt = tiles128 >= 2 * 148 ? 128 : 64;
+        bt = tiles128 >= 2 * dev->sms ? 128 : 64;
     }
     dim3 grid(cdiv(p.N, bt), cdiv(p.M, bt), p.ksplit > 1 ? p.ksplit : batches);
     if (grid_out) *grid_out = grid;          // the tile grid (what the partials are indexed by)

@@ -601,17 +601,14 @@ inline int make_slice_map(CUtensorMap* m, int8_t* Q, int cols_pad, int n_pad, in
 
 inline int gram_accumulate(double* H, GramSource src, int cols, int n, void* ws, int32_t* status,
                            cudaStream_t stream) {
-    static bool attr_done = false;
-    static int num_sms = 0;
-    if (!attr_done) {
-        if (cudaFuncSetAttribute(gram_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGramSmemBytes) !=
-            cudaSuccess)
-            return PTQ_ERR_CUDA;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-        attr_done = true;
-    }
+    DeviceState* dev = nullptr;
+    int dst = current_device_state(&dev);
+    if (dst) return dst;
+    dst = ensure_smem_attr(dev, SA_GRAM, [] {
+        return cudaFuncSetAttribute(gram_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kGramSmemBytes);
+    });
+    if (dst) return dst;
+    const int num_sms = dev->sms;
     const int cols_pad = cdiv(cols, 128) * 128;
     const int max_chunk = n < kGramMaxChunk ? n : kGramMaxChunk;
     const size_t n_pad_max = (size_t)cdiv(max_chunk, 128) * 128;

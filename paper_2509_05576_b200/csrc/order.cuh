@@ -104,18 +104,21 @@ __device__ __forceinline__ unsigned long long sortable_key(double x) {
     return (u & 0x8000000000000000ull) ? ~u : (u | 0x8000000000000000ull);
 }
 
-// perm[rank_j] = j with rank_j = #{k : S_k > S_j, or S_k == S_j and k < j}: a stable descending sort by counting.
+// perm[rank_j] = j with rank_j = #{k : S_k > S_j, or S_k == S_j and k < j}: a stable descending sort by counting
+// (ascending != 0: S_k < S_j instead, the "asc" keys of Sec. 4.1; equal scores keep the lower index first either way).
 // 32 columns j per CTA; the eight lanes that share a column each count a strided eighth of the keys.
 constexpr int kRankCols = 32;
-__global__ void __launch_bounds__(256) rank_sort_kernel(const double* __restrict__ S, int cols,
+__global__ void __launch_bounds__(256) rank_sort_kernel(const double* __restrict__ S, int cols, int ascending,
                                                          int32_t* __restrict__ perm) {
     __shared__ unsigned long long keys[1024];
     const int j = blockIdx.x * kRankCols + (threadIdx.x >> 3);
     const int part = threadIdx.x & 7;
-    const unsigned long long kj = j < cols ? sortable_key(S[j]) : 0ull;
+    // ascending order is descending order of the complemented keys
+    const unsigned long long flip = ascending ? ~0ull : 0ull;
+    const unsigned long long kj = j < cols ? (sortable_key(S[j]) ^ flip) : 0ull;
     int rank = 0;
     for (int t0 = 0; t0 < cols; t0 += 1024) {
-        for (int t = threadIdx.x; t < 1024; t += 256) keys[t] = t0 + t < cols ? sortable_key(S[t0 + t]) : 0ull;
+        for (int t = threadIdx.x; t < 1024; t += 256) keys[t] = t0 + t < cols ? (sortable_key(S[t0 + t]) ^ flip) : 0ull;
         __syncthreads();
         const int lim = min(1024, cols - t0);
         for (int t = part; t < lim; t += 8) {

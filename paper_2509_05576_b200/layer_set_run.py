@@ -49,6 +49,73 @@ def stage_work(spec):
     }
 
 
+def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP64_PEAK_TFLOPS, ws=None, flush=None):
+    """Quantizes the given layers one after the other on the current stream and times every C-ABI call with CUDA
+    events (L2 flushed before every timed repetition, median over the repetitions).  Consecutive specs that describe
+    the same seeded layer at another bit-width reuse its inputs.  Returns the per-layer records, the set totals, the
+    per-stage totals and the per-stage roofline fractions of the whole set (sum of work / sum of time / peak)."""
+    hbm, bf16, src = _peaks()
+    int8_peak = bf16 * INT8_OVER_BF16
+    s = torch.cuda.current_stream()
+    flush = flush if flush is not None else torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
+    ws = ws or ptq.Workspace()
+    rows_out = []
+    totals = {"weights": 0, "ms": 0.0, "loss": 0.0}
+    stage_tot, work_tot = {}, {}
+    if not quiet:
+        print(f"{'layer':28s} {'rows':>5s} {'cols':>6s} {'n':>5s} {'b':>2s} {'total ms':>9s} {'Mw/s':>8s} "
+              f"{'hess':>7s} {'inv':>7s} {'order':>6s} {'sweep':>7s} {'%int8':>6s} {'%f64 inv':>8s} {'%f64 swp':>8s} {'loss':>12s}")
+    key, Wd, Xd, bufs = None, None, None, None
+    for spec in specs:
+        k = (spec.rows, spec.cols, spec.n, spec.w_dist, spec.x_dist, spec.seed)
+        if k != key:
+            Wd = Xd = bufs = None
+            W, X = wl.make_layer(spec)
+            Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
+            bufs = ptq.LayerBuffers(spec.rows, spec.cols)
+            key = k
+        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=score_mode, bufs=bufs, ws=ws, stream=s)    # warm-up
+        torch.cuda.synchronize()
+        ptq.check_status(bufs.status, spec.name)
+        per = {}
+        for rep in range(reps):
+            flush.fill_(rep)
+            ev = []
+            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=score_mode, bufs=bufs, ws=ws, stream=s, events=ev)
+            torch.cuda.synchronize()
+            for name, a, b in ev:
+                per.setdefault(name, []).append(a.elapsed_time(b))
+        ptq.check_status(bufs.status, spec.name)
+        st = {k2: float(np.median(v)) for k2, v in per.items()}
+        total = sum(st.values())
+        work = stage_work(spec)
+        frac = {"hessian": work["hessian"] / (st["hessian"] * 1e-3) / 1e12 / int8_peak,
+                "inverse": work["inverse"] / (st["inverse"] * 1e-3) / 1e12 / fp64_peak,
+                "sweep": work["sweep"] / (st["sweep"] * 1e-3) / 1e12 / fp64_peak}
+        loss = float(bufs.loss.item())
+        if not quiet:
+            print(f"{spec.name:28s} {spec.rows:5d} {spec.cols:6d} {spec.n:5d} {spec.bits:2d} {total:9.3f} "
+                  f"{spec.weights / total / 1e3:8.1f} {st['hessian']:7.3f} {st['inverse']:7.3f} "
+                  f"{st['grid'] + st['order']:6.3f} {st['sweep']:7.3f} {100 * frac['hessian']:6.2f} "
+                  f"{100 * frac['inverse']:8.2f} {100 * frac['sweep']:8.2f} {loss:12.5g}")
+        rows_out.append({"layer": spec.name, "rows": spec.rows, "cols": spec.cols, "n": spec.n, "bits": spec.bits,
+                         "ms": total, "stages_ms": st, "roofline_frac": frac, "loss": loss})
+        totals["weights"] += spec.weights
+        totals["ms"] += total
+        totals["loss"] += loss
+        for k2, v in st.items():
+            stage_tot[k2] = stage_tot.get(k2, 0.0) + v
+        for k2, v in work.items():
+            work_tot[k2] = work_tot.get(k2, 0.0) + v
+    stage_frac = {"hessian": work_tot["hessian"] / (stage_tot["hessian"] * 1e-3) / 1e12 / int8_peak,
+                  "inverse": work_tot["inverse"] / (stage_tot["inverse"] * 1e-3) / 1e12 / fp64_peak,
+                  "sweep": work_tot["sweep"] / (stage_tot["sweep"] * 1e-3) / 1e12 / fp64_peak}
+    return {"layers": rows_out, "n_layers": len(rows_out), "weights": totals["weights"], "total_ms": totals["ms"],
+            "weights_per_s": totals["weights"] / (totals["ms"] * 1e-3), "loss_sum": totals["loss"],
+            "stage_total_ms": stage_tot, "stage_roofline_frac": stage_frac,
+            "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak, "fp64_tflops": fp64_peak, "source": src}}
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7])
@@ -61,6 +128,7 @@ def main(argv=None):
                          "(inputs resident, nothing synchronised in between) and report the wall time of that")
     ap.add_argument("--score-mode", default="qerr", choices=sorted(SCORE_MODES),
                     help="column ordering: qerr (Eq. 10, the method's), prune (Eq. 8), err, w, none (no sorting)")
+    ap.add_argument("--ascending", action="store_true", help="sort the scores ascending (the 'asc' keys of Sec. 4.1)")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise RuntimeError("layer_set_run needs a CUDA device")
@@ -74,52 +142,11 @@ def main(argv=None):
         specs = [s for s in specs if s.cols <= args.max_cols]
     if args.limit:
         specs = specs[:args.limit]
-    hbm, bf16, src = _peaks()
-    int8_peak = bf16 * INT8_OVER_BF16
     s = torch.cuda.current_stream()
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
-    ws = ptq.Workspace()
-    rows_out = []
-    totals = {"weights": 0, "ms": 0.0, "loss": 0.0}
-    stage_tot = {}
-    print(f"{'layer':28s} {'rows':>5s} {'cols':>6s} {'n':>5s} {'b':>2s} {'total ms':>9s} {'Mw/s':>8s} "
-          f"{'hess':>7s} {'inv':>7s} {'order':>6s} {'sweep':>7s} {'%int8':>6s} {'%f64 inv':>8s} {'%f64 swp':>8s} {'loss':>12s}")
-    for spec in specs:
-        W, X = wl.make_layer(spec)
-        Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
-        bufs = ptq.LayerBuffers(spec.rows, spec.cols)
-        mode = SCORE_MODES[args.score_mode]
-        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=mode, bufs=bufs, ws=ws, stream=s)    # warm-up
-        torch.cuda.synchronize()
-        ptq.check_status(bufs.status, spec.name)
-        per = {}
-        for rep in range(args.reps):
-            flush.fill_(rep)
-            ev = []
-            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=mode, bufs=bufs, ws=ws, stream=s, events=ev)
-            torch.cuda.synchronize()
-            for name, a, b in ev:
-                per.setdefault(name, []).append(a.elapsed_time(b))
-        ptq.check_status(bufs.status, spec.name)
-        st = {k: float(np.median(v)) for k, v in per.items()}
-        total = sum(st.values())
-        work = stage_work(spec)
-        frac = {"hessian": work["hessian"] / (st["hessian"] * 1e-3) / 1e12 / int8_peak,
-                "inverse": work["inverse"] / (st["inverse"] * 1e-3) / 1e12 / FP64_PEAK_TFLOPS,
-                "sweep": work["sweep"] / (st["sweep"] * 1e-3) / 1e12 / FP64_PEAK_TFLOPS}
-        loss = float(bufs.loss.item())
-        print(f"{spec.name:28s} {spec.rows:5d} {spec.cols:6d} {spec.n:5d} {spec.bits:2d} {total:9.3f} "
-              f"{spec.weights / total / 1e3:8.1f} {st['hessian']:7.3f} {st['inverse']:7.3f} "
-              f"{st['grid'] + st['order']:6.3f} {st['sweep']:7.3f} {100 * frac['hessian']:6.2f} "
-              f"{100 * frac['inverse']:8.2f} {100 * frac['sweep']:8.2f} {loss:12.5g}")
-        rows_out.append({"layer": spec.name, "rows": spec.rows, "cols": spec.cols, "n": spec.n, "bits": spec.bits,
-                         "ms": total, "stages_ms": st, "roofline_frac": frac, "loss": loss})
-        totals["weights"] += spec.weights
-        totals["ms"] += total
-        totals["loss"] += loss
-        for k, v in st.items():
-            stage_tot[k] = stage_tot.get(k, 0.0) + v
-        del Wd, Xd, bufs
+    mode = SCORE_MODES[args.score_mode] | (ptq.SCORE_ASCENDING if args.ascending else 0)
+    res = run_specs(specs, args.reps, mode, quiet=False, flush=flush)
+    totals = {"ms": res["total_ms"]}
     overlapped = None
     if args.streams > 1:
         # independent layers on several streams: every stream has its own workspace and output buffers; the inputs
@@ -135,7 +162,7 @@ def main(argv=None):
         def run_set():
             for i, (spec, Wd, Xd) in enumerate(data):
                 k = i % len(streams)
-                ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=SCORE_MODES[args.score_mode],
+                ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=mode,
                                         bufs=outs[i], ws=wss[k], stream=streams[k])
 
         times = []
@@ -159,12 +186,12 @@ def main(argv=None):
                       "loss_sum": float(sum(o.loss.item() for o in outs))}
         print(f"whole set on {args.streams} streams: {overlapped['set_ms']:.2f} ms "
               f"(sum of the per-layer times on one stream: {totals['ms']:.2f} ms)")
-    print(json.dumps({"config": args.config, "score_mode": args.score_mode, "loss_sum": totals["loss"],
-                      "overlapped": overlapped,
-                      "layers": len(rows_out), "weights": totals["weights"],
-                      "total_ms": totals["ms"], "weights_per_s": totals["weights"] / (totals["ms"] * 1e-3),
-                      "stage_total_ms": stage_tot, "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak,
-                                                             "fp64_tflops": FP64_PEAK_TFLOPS, "source": src}}))
+    print(json.dumps({"config": args.config, "score_mode": args.score_mode, "ascending": bool(args.ascending),
+                      "loss_sum": res["loss_sum"], "overlapped": overlapped,
+                      "layers": res["n_layers"], "weights": res["weights"],
+                      "total_ms": res["total_ms"], "weights_per_s": res["weights_per_s"],
+                      "stage_total_ms": res["stage_total_ms"], "stage_roofline_frac": res["stage_roofline_frac"],
+                      "peaks": res["peaks"]}))
     return 0
 
 

@@ -20,10 +20,12 @@ ERR_STATIC_SCRATCH = 9
 STATIC_SCRATCH_BYTES = 6 << 20
 DAMP_REL_MEAN_DIAG, DAMP_ABS = 0, 1
 SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
+SCORE_ASCENDING = 16          # added to a score mode: sort by S ascending
 CALL_HESSIAN_ACCUMULATE, CALL_PREPARE_HINV, CALL_SENSITIVITY_ORDER, CALL_QUANTIZE_LAYER, CALL_HESSIAN_ACCUMULATE_F64 = range(5)
 
 EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_conv", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
            "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_sensitivity_order_static", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
+           "ptq_sort_scores", "ptq_selftest_wait_timeout", "ptq_fp64_probe",
            "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
 
 
@@ -62,6 +64,9 @@ def lib():
         L.ptq_sensitivity_order_static.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, vp]
         L.ptq_quantize_layer.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, vp, c_int, vp, vp, vp, vp, vp,
                                          c_size_t, vp, vp]
+        L.ptq_sort_scores.argtypes = [vp, c_int, c_int, vp, vp]
+        L.ptq_selftest_wait_timeout.argtypes = [c_int, ctypes.c_longlong, vp, c_size_t, vp, vp]
+        L.ptq_fp64_probe.argtypes = [c_int, c_int, vp, ctypes.POINTER(c_double), vp]
         L.ptq_status_string.argtypes = [c_int]
         L.ptq_status_string.restype = ctypes.c_char_p
         L.ptq_version.restype = c_int
@@ -230,6 +235,28 @@ def sensitivity_order_static(W, Hinv_diag, scale, zero, bits, score_mode, S, per
     _check(lib().ptq_sensitivity_order_static(_ptr(W), rows, cols, _rowmajor(W, "W"), _ptr(Hinv_diag), _ptr(scale),
                                               _ptr(zero), int(bits), int(score_mode), _ptr(S), _ptr(perm),
                                               _ptr(status), _stream(stream)), "ptq_sensitivity_order_static")
+
+
+def sort_scores(S, perm, ascending=False, stream=None):
+    """perm = indices sorted by S descending (or ascending), stable (Sec. 4.2 step 3)."""
+    _dev(S, torch.float64, "S"); _dev(perm, torch.int32, "perm")
+    _check(lib().ptq_sort_scores(_ptr(S), S.numel(), 1 if ascending else 0, _ptr(perm), _stream(stream)),
+           "ptq_sort_scores")
+
+
+def selftest_wait_timeout(which, limit_cycles, ws, status, stream=None):
+    """Makes one of the library's bounded device-side waits run out (0: grid barrier, 1: sweep counter)."""
+    buf = ws.get(256)
+    _check(lib().ptq_selftest_wait_timeout(int(which), int(limit_cycles), _ptr(buf), buf.numel(), _ptr(status),
+                                           _stream(stream)), "ptq_selftest_wait_timeout")
+
+
+def fp64_probe(kind, iters, sink, stream=None) -> float:
+    """Launches the float64 throughput probe (0: FMA, 1: tensor-core MMA); returns the flops of that launch."""
+    flops = c_double(0.0)
+    _check(lib().ptq_fp64_probe(int(kind), int(iters), _ptr(sink), ctypes.byref(flops), _stream(stream)),
+           "ptq_fp64_probe")
+    return flops.value
 
 
 def quantize_layer(W, Hinv, perm, scale, zero, bits, codes, What, H_undamped, loss_out, ws, status, stream=None):

@@ -78,6 +78,29 @@ def test_bad_arguments_are_rejected_on_the_host(lib):
                                   fake, None) == ptq.ERR_WORKSPACE
 
 
+def test_new_entry_points_check_their_arguments_on_the_host(lib):
+    from paper_2509_05576_b200 import ptq
+    vp = ctypes.c_void_p
+    fake = vp(4096)
+    assert lib.ptq_sort_scores(None, 8, 0, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_sort_scores(fake, 0, 0, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_selftest_wait_timeout(2, 1000, fake, 64, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_selftest_wait_timeout(0, 0, fake, 64, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_selftest_wait_timeout(0, 10 ** 12, fake, 64, fake, None) == ptq.ERR_INVALID_ARG   # beyond the library's own limit
+    assert lib.ptq_selftest_wait_timeout(0, 1000, fake, 8, fake, None) == ptq.ERR_WORKSPACE
+    flops = ctypes.c_double(0.0)
+    assert lib.ptq_fp64_probe(2, 10, fake, ctypes.byref(flops), None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_fp64_probe(0, 0, fake, ctypes.byref(flops), None) == ptq.ERR_INVALID_ARG
+    # score modes: a direction flag on a valid mode is accepted by the argument check, anything else is not
+    args = (fake, 4, 4, 4, fake, fake, fake, 4)
+    assert lib.ptq_sensitivity_order(*args, 5, fake, fake, fake, 1 << 20, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_sensitivity_order(*args, 32, fake, fake, fake, 1 << 20, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_sensitivity_order(*args, ptq.SCORE_W | ptq.SCORE_ASCENDING, fake, fake, None, 0, fake, None) == ptq.ERR_WORKSPACE
+    # sizes beyond what the launch grid can index are refused, not launched
+    assert lib.ptq_quantize_layer(fake, 70000, 8, 8, fake, fake, fake, fake, 4, fake, None, None, None, fake, 1 << 40,
+                                  fake, None) == ptq.ERR_UNSUPPORTED
+
+
 def test_binding_refuses_cpu_tensors(lib):
     import torch
     from paper_2509_05576_b200 import ptq

@@ -149,3 +149,60 @@ def test_more_block_rows_than_sms():
     rtn = sc[:, None] * (torch.clamp(torch.round(Wd / sc[:, None]) + zp[:, None], 0, 2 ** bits - 1) - zp[:, None])
     dR = Wd - rtn.float().double()
     assert loss_def < 0.5 * float(((dR @ H) * dR).sum())
+
+
+def test_largest_scaling_shape_4096x11008_all_bit_widths():
+    """The widest benchmark layer (11008 columns against 8192 calibration columns), at 3, 4 and 8 bits.
+
+    Hessian, damped inverse, scores and column order are compared with the oracle in full.  The literal Eq. 12 loop
+    is out of reach at this width (4.4e11 multiply-adds per pass over a 970 MB matrix), so the sweep is checked with
+    the oracle's factor-form mode -- pinned equal to the literal loop on every width that loop reaches
+    (tests/test_oracle_pins.py) -- on 32 seeded rows, which are independent of the other rows once the order and the
+    inverse Hessian are fixed (Sec. 4.2 step 4)."""
+    specs = wl.config5(bits=(3, 4, 8), shapes=((4096, 11008),))
+    W, X = wl.make_layer(specs[0])
+    cols = specs[0].cols
+    H = oracle.hessian_accumulate(X)
+    Hinv, diag, lam = oracle.prepare_hinv(H, specs[0].damp)
+    Wd, Xd = torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()
+    Hd = torch.from_numpy(H).cuda()
+    bufs, ws = ptq.LayerBuffers(specs[0].rows, cols), ptq.Workspace()
+    for k, spec in enumerate(specs):
+        Wk, Xk = (W, X) if k == 0 else wl.make_layer(spec)
+        assert np.array_equal(Wk, W) and np.array_equal(Xk, X)               # one layer, three bit-widths
+        ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, bufs=bufs, ws=ws)
+        torch.cuda.synchronize()
+        ptq.check_status(bufs.status, spec.name)
+        if k == 0:
+            assert float((bufs.H - Hd).abs().max()) <= 2e-12 * float(np.max(np.abs(H)))
+            gHinv = bufs.Hinv.cpu().numpy()
+            assert np.max(np.abs(gHinv - Hinv)) <= 1e-9 * np.max(np.abs(Hinv))
+            assert abs(float(bufs.lam.item()) - lam) <= 2e-12 * lam          # lambda follows the GPU's own H
+            del gHinv
+        sc, zp = oracle.minmax_grid(W, spec.bits)
+        assert np.array_equal(bufs.scale.cpu().numpy(), sc) and np.array_equal(bufs.zero.cpu().numpy(), zp)
+        S, perm = oracle.sensitivity_order(W, diag, sc, zp, spec.bits)
+        assert np.allclose(bufs.S.cpu().numpy(), S, rtol=1e-9, atol=0)
+        assert np.array_equal(bufs.perm.cpu().numpy(), perm), "column order differs"
+        U = oracle.factor_upper(Hinv, perm)
+        rows = np.sort(np.random.Generator(np.random.PCG64(spec.seed + spec.bits)).choice(spec.rows, 32, replace=False))
+        ref = oracle.quantize_rows_factor(W[rows], U, perm, sc[rows], zp[rows], spec.bits, want_prer=True)
+        del U
+        ref["perm"] = perm
+        g_codes, g_What = bufs.codes.cpu().numpy(), bufs.What.cpu().numpy()
+        nm = compare_codes(g_codes[rows], ref)
+        if nm == 0:
+            assert np.array_equal(g_What[rows], ref["What"])
+        num = np.linalg.norm(g_What[rows].astype(np.float64) - ref["What"].astype(np.float64))
+        assert num <= WHAT_RTOL * np.linalg.norm(ref["What"].astype(np.float64))
+        assert g_codes.max() <= 2 ** spec.bits - 1
+        # loss against its definition, 1/2 tr(dW H dW^T), with the GPU's own What (library matmul on the device)
+        dW = Wd.double() - bufs.What.double()
+        loss_def = 0.5 * float(((dW @ Hd) * dW).sum())
+        assert abs(float(bufs.loss.item()) - loss_def) <= 1e-9 * loss_def
+        # and on the oracle's rows: the oracle's What gives the same per-row loss as the GPU's
+        dWs = W[rows].astype(np.float64) - ref["What"].astype(np.float64)
+        loss_rows = 0.5 * float(np.sum((dWs @ H) * dWs))
+        dWg = dW[torch.from_numpy(rows).cuda()]
+        assert abs(0.5 * float(((dWg @ Hd) * dWg).sum()) - loss_rows) <= LOSS_RTOL * loss_rows
+        del dW, dWg

@@ -175,6 +175,57 @@ def test_scores_and_order_match_oracle(mode, rows, cols):
     assert np.array_equal(perm.cpu().numpy(), ref_perm)
 
 
+@pytest.mark.parametrize("mode", [ptq.SCORE_QERR, ptq.SCORE_PRUNE, ptq.SCORE_ERR, ptq.SCORE_W])
+def test_ascending_order_matches_oracle_and_whole_path(mode):
+    """The "asc" keys of Sec. 4.1: same scores, ascending stable order; then the whole path in that order."""
+    W, X = _layer(70, 333, 400, 471)
+    W[:, 17] = W[:, 3]
+    H = oracle.hessian_accumulate(X)
+    Hinv, diag, _ = oracle.prepare_hinv(H)
+    diag[17] = diag[3]
+    sc, zp = oracle.minmax_grid(W, 4)
+    ref_S, ref_perm = oracle.sensitivity_order(W, diag, sc, zp, 4, mode | oracle.SCORE_ASCENDING)
+    S = torch.empty(333, dtype=torch.float64, device="cuda")
+    perm = torch.empty(333, dtype=torch.int32, device="cuda")
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.sensitivity_order(_cuda(W), _cuda(diag), _cuda(sc), _cuda(zp), 4, mode | ptq.SCORE_ASCENDING, S, perm, ws, st)
+    # the sort alone, from scores the caller already has
+    perm2 = torch.empty(333, dtype=torch.int32, device="cuda")
+    ptq.sort_scores(S, perm2, ascending=True)
+    perm3 = torch.empty(333, dtype=torch.int32, device="cuda")
+    ptq.sort_scores(S, perm3, ascending=False)
+    torch.cuda.synchronize()
+    ptq.check_status(st)
+    assert np.allclose(S.cpu().numpy(), ref_S, rtol=1e-13, atol=0)
+    assert np.array_equal(perm.cpu().numpy(), ref_perm)
+    assert np.array_equal(perm2.cpu().numpy(), ref_perm)
+    _, ref_desc = oracle.sensitivity_order(W, diag, sc, zp, 4, mode)
+    assert np.array_equal(perm3.cpu().numpy(), ref_desc)
+    ref = oracle_layer(W, X, 4, score_mode=mode | oracle.SCORE_ASCENDING)
+    g = gpu_layer(W, X, 4, score_mode=mode | ptq.SCORE_ASCENDING)
+    assert assert_layer_parity(g, ref) == 0
+
+
+# ------------------------------------------------------------------------------------------ bounded waits
+@pytest.mark.parametrize("which", [0, 1])
+def test_bounded_wait_runs_out_and_the_context_stays_usable(which):
+    """The factorisation's grid barrier (0) and the sweep's counter wait (1) are asked, with a limit of a few thousand
+    cycles, for something that never comes: the kernel must return with PTQ_ERR_TIMEOUT in the status word, and an
+    ordinary call made afterwards on the same stream must give exactly what it gave before."""
+    W, X = _layer(48, 200, 300, 480)
+    before = gpu_layer(W, X, 4)
+    st, ws = ptq.new_status(), ptq.Workspace()
+    ptq.selftest_wait_timeout(which, 5000, ws, st)
+    torch.cuda.synchronize()
+    with pytest.raises(ptq.PtqError) as ei:
+        ptq.check_status(st)
+    assert ei.value.code == ptq.ERR_TIMEOUT
+    assert int(st.cpu()[2]) == 1 + which
+    after = gpu_layer(W, X, 4)
+    for k in ("H", "Hinv", "S", "perm", "codes", "What", "loss"):
+        assert np.array_equal(before[k], after[k]), k
+
+
 # ------------------------------------------------------------------------------------------ column sweep
 def _sweep(W, Hinv, perm, sc, zp, bits, H=None):
     rows, cols = W.shape
@@ -287,3 +338,33 @@ def test_config2_full_size():
     assert np.max(np.abs(g["Hinv"] - ref["Hinv"])) <= 1e-10 * np.max(np.abs(ref["Hinv"]))
     assert_layer_parity(g, ref)
     assert abs(float(g["loss"][0]) - oracle.loss_direct(W, g["What"], X)) <= 1e-9 * ref["loss"]
+
+
+def test_sharded_entry_on_one_rank_equals_the_single_gpu_path():
+    """The multi-GPU entry (all-reduce of H over the calibration split, of the scores over the row split) on a group
+    of one NCCL rank: the collectives are no-ops, so the result must be that of the ordinary path, bit for bit, and
+    match the oracle.  (More ranks need more GPUs; the sharding logic itself runs as gloo ranks in the CPU suite.)"""
+    import os
+    import socket
+    import torch.distributed as dist
+    from paper_2509_05576_b200 import sharded
+    W, X = _layer(70, 200, 300, 990)
+    ref = oracle_layer(W, X, 4)
+    g = gpu_layer(W, X, 4)
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        ops = sharded.GpuOps()
+        res = sharded.quantize_layer_sharded(_cuda(W), _cuda(X), 200, 4, ops=ops)
+        torch.cuda.synchronize()
+        ops.check()
+    finally:
+        dist.destroy_process_group()
+    for k in ("H", "Hinv", "S", "perm", "codes", "What"):
+        assert np.array_equal(res[k].cpu().numpy(), g[k]), k
+    assert float(res["loss"].item()) == float(g["loss"][0])
+    out = {k: res[k].cpu().numpy() for k in ("perm", "scale", "zero", "codes", "What", "loss")}
+    assert assert_layer_parity(out, ref) == 0

@@ -48,8 +48,11 @@ def _both(rows, cols, seed, bits, mode):
 
 
 def test_static_variant_matches_workspace_variant_on_two_calls_in_a_row():
-    # first call: several row chunks and a ragged last one; second call: a smaller, differently shaped problem
-    for rows, cols, seed, bits, mode in [(200, 333, 21, 4, ptq.SCORE_QERR), (70, 129, 22, 3, ptq.SCORE_PRUNE)]:
+    # first call: several row chunks and a ragged last one; second call: a smaller, differently shaped problem; then
+    # the ascending order and the identity order (no sorting), which reads nothing from the array
+    for rows, cols, seed, bits, mode in [(200, 333, 21, 4, ptq.SCORE_QERR), (70, 129, 22, 3, ptq.SCORE_PRUNE),
+                                         (90, 77, 23, 4, ptq.SCORE_ERR | ptq.SCORE_ASCENDING),
+                                         (33, 50, 24, 4, ptq.SCORE_NONE)]:
         S_ref, p_ref, S, p = _both(rows, cols, seed, bits, mode)
         # same kernels, same summation order: the scores agree to the tolerance of the score parity test (and in
         # fact bit for bit), the order exactly
@@ -57,6 +60,26 @@ def test_static_variant_matches_workspace_variant_on_two_calls_in_a_row():
         assert np.array_equal(S, S_ref)
         assert np.array_equal(p, p_ref)
         assert sorted(p.tolist()) == list(range(cols))
+
+
+def test_static_variant_allocates_nothing_and_takes_a_problem_exactly_at_the_limit():
+    # 96 row chunks x 8192 columns x 8 bytes is exactly the size of the built-in array: accepted
+    rows, cols, bits = 96 * 64, 8192, 4
+    assert (rows // 64) * cols * 8 == ptq.STATIC_SCRATCH_BYTES
+    Wd, diag, scale, zero, st = _inputs(rows, cols, 25, bits)
+    S_ref = torch.empty(cols, dtype=torch.float64, device="cuda")
+    p_ref = torch.empty(cols, dtype=torch.int32, device="cuda")
+    ptq.sensitivity_order(Wd, diag, scale, zero, bits, ptq.SCORE_QERR, S_ref, p_ref, ptq.Workspace(), st)
+    S = torch.empty(cols, dtype=torch.float64, device="cuda")
+    p = torch.empty(cols, dtype=torch.int32, device="cuda")
+    ptq.sensitivity_order_static(Wd, diag, scale, zero, bits, ptq.SCORE_QERR, S, p, st)     # first call: module set-up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    ptq.sensitivity_order_static(Wd, diag, scale, zero, bits, ptq.SCORE_QERR, S, p, st)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before       # the device's free memory did not move
+    ptq.check_status(st, "sensitivity_order_static")
+    assert torch.equal(S, S_ref) and torch.equal(p, p_ref)
 
 
 def test_static_variant_refuses_what_does_not_fit():
