@@ -70,7 +70,8 @@ typedef enum {
     PTQ_CALL_PREPARE_HINV = 1,
     PTQ_CALL_SENSITIVITY_ORDER = 2,
     PTQ_CALL_QUANTIZE_LAYER = 3,
-    PTQ_CALL_HESSIAN_ACCUMULATE_F64 = 4
+    PTQ_CALL_HESSIAN_ACCUMULATE_F64 = 4,
+    PTQ_CALL_QUANTIZE_LAYER_DYNAMIC = 5
 } ptq_call_id;
 
 /* Minimum workspace, in bytes, for one call with these sizes (host function, no CUDA calls). */
@@ -178,6 +179,23 @@ int ptq_quantize_layer(const float *W, int rows, int cols, int64_t ldw, const do
                        const float *scale, const float *zero, int bits, uint8_t *codes, float *What,
                        const double *H_undamped, double *loss_out, void *ws, size_t ws_bytes, int32_t *status,
                        void *stream);
+
+/*
+ * The column loop with dynamic re-ranking.  Sec. 5 writes the sort inside the per-column loop; read literally, the
+ * columns still to be quantized are ranked again while the loop runs.  Every `block` columns the scores of the
+ * REMAINING columns are recomputed from the current (compensated) weights and the diagonal of the current
+ * (Eq.-12-updated) inverse Hessian, the remaining columns are sorted by them (keys, direction and tie rule of
+ * ptq_sensitivity_order; ties by ORIGINAL column index) and the next `block` columns are quantized in that order
+ * with Eq. 11 / Eq. 12.  block >= cols is ptq_sensitivity_order followed by ptq_quantize_layer.
+ *   block      a multiple of 64, or >= cols (PTQ_ERR_UNSUPPORTED otherwise)
+ *   order_out  [cols] int32, out: the sequence in which the columns were quantized
+ *   other arguments as for ptq_quantize_layer (outputs in original column order); Hinv_diag is not needed
+ * Workspace: ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER_DYNAMIC, rows, cols, 0).
+ */
+int ptq_quantize_layer_dynamic(const float *W, int rows, int cols, int64_t ldw, const double *Hinv, const float *scale,
+                               const float *zero, int bits, int score_mode, int block, uint8_t *codes, float *What,
+                               int32_t *order_out, const double *H_undamped, double *loss_out, void *ws,
+                               size_t ws_bytes, int32_t *status, void *stream);
 
 /*
  * Sec. 4.2 step 3 alone: perm = the indices 0 .. cols-1 sorted by S descending (ascending != 0: ascending), equal

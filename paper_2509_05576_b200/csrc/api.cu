@@ -5,6 +5,7 @@
 #include "order.cuh"
 #include "colloop.cuh"
 #include "gram.cuh"
+#include "dynamic.cuh"
 
 using namespace ptq;
 
@@ -59,8 +60,8 @@ int order_launch(const float* W, int rows, int cols, int64_t ldw, const double* 
     if (chunks > 65535) return PTQ_ERR_UNSUPPORTED;
     if (mode != PTQ_SCORE_NONE) {
         Launch l(K_SCORE_PARTIAL, stream);
-        score_partial_kernel<<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero, bits,
-                                                                              mode, partial);
+        score_partial_kernel<float><<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero,
+                                                                                     bits, mode, partial);
     }
     { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, mode, S, status); }
     { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, ascending, perm); }
@@ -216,6 +217,26 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(((size_t)cdiv(rows, kSweepRows) + 1) * sizeof(unsigned));   // per-row-group progress counters of the sweep
             add(chol_scratch_doubles(cols) * sizeof(double));
             break;
+        case PTQ_CALL_QUANTIZE_LAYER_DYNAMIC:
+            if (rows < 1) return 0;
+            add(c * c * sizeof(double));                    // current matrix and the gathered one (ping-pong)
+            add(c * c * sizeof(double));
+            add((size_t)rows * c * sizeof(double));         // current weights and the gathered ones (ping-pong)
+            add((size_t)rows * c * sizeof(double));
+            add((size_t)rows * c * sizeof(double));         // scaled errors E
+            add((size_t)rows * c * sizeof(double));         // dW
+            add((size_t)rows * c);                          // codes of the block being swept
+            add(c * sizeof(double));                        // scores
+            add(c * sizeof(double));                        // diagonal
+            add((size_t)cdiv(rows, kScoreRowChunk) * c * sizeof(double));
+            add(c * sizeof(int32_t));                       // order of the round
+            add(c * sizeof(int32_t));                       // original column of every position (ping-pong)
+            add(c * sizeof(int32_t));
+            add(loss_partials_count(rows, cols) * sizeof(double));
+            add(2 * sizeof(unsigned));
+            add(((size_t)cdiv(rows, kSweepRows) + 1) * sizeof(unsigned));
+            add(chol_scratch_doubles(cols) * sizeof(double));
+            break;
         default:
             return 0;
     }
@@ -335,6 +356,124 @@ int ptq_sensitivity_order_static(const float* W, int rows, int cols, int64_t ldw
     // left in the array by an earlier call is ever used and nothing needs clearing.
     return order_launch(W, rows, cols, ldw, Hinv_diag, scale, zero, bits, score_mode & ~PTQ_SCORE_ASCENDING,
                         (score_mode & PTQ_SCORE_ASCENDING) ? 1 : 0, S, perm, partial, status, stream);
+}
+
+int ptq_quantize_layer_dynamic(const float* W, int rows, int cols, int64_t ldw, const double* Hinv, const float* scale,
+                               const float* zero, int bits, int score_mode, int block, uint8_t* codes, float* What,
+                               int32_t* order_out, const double* H_undamped, double* loss_out, void* ws,
+                               size_t ws_bytes, int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!W || !Hinv || !scale || !zero || !codes || !order_out || rows < 1 || cols < 1 || ldw < cols || bits < 2 ||
+        bits > 8 || block < 1)
+        return PTQ_ERR_INVALID_ARG;
+    if (score_mode & ~(PTQ_SCORE_ASCENDING | 7)) return PTQ_ERR_INVALID_ARG;
+    const int mode = score_mode & ~PTQ_SCORE_ASCENDING, ascending = (score_mode & PTQ_SCORE_ASCENDING) ? 1 : 0;
+    if (mode < PTQ_SCORE_QERR || mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
+    if (block < cols && (block % kNB) != 0) return PTQ_ERR_UNSUPPORTED;     // rounds end on the 64-column block grid
+    if (rows > kMaxGridY || cols > kMaxGridY || cdiv(rows, kScoreRowChunk) > kMaxGridY) return PTQ_ERR_UNSUPPORTED;
+    if (!aligned16(Hinv) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER_DYNAMIC, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
+    const size_t c = (size_t)cols;
+    Carver cv(ws);
+    double* Abuf[2] = {cv.take<double>(c * c), nullptr};
+    Abuf[1] = cv.take<double>(c * c);
+    double* Wbuf[2] = {cv.take<double>((size_t)rows * c), nullptr};
+    Wbuf[1] = cv.take<double>((size_t)rows * c);
+    double* E = cv.take<double>((size_t)rows * c);
+    double* dW = cv.take<double>((size_t)rows * c);
+    uint8_t* codes_p = cv.take<uint8_t>((size_t)rows * c);
+    double* S = cv.take<double>(c);
+    double* diag = cv.take<double>(c);
+    const int chunks = cdiv(rows, kScoreRowChunk);
+    double* partial = cv.take<double>((size_t)chunks * c);
+    int32_t* ordr = cv.take<int32_t>(c);
+    int32_t* obuf[2] = {cv.take<int32_t>(c), nullptr};
+    obuf[1] = cv.take<int32_t>(c);
+    double* partials = cv.take<double>(loss_partials_count(rows, cols));
+    unsigned* bar = cv.take<unsigned>(2);
+    unsigned* sweep_flags = cv.take<unsigned>((size_t)cdiv(rows, kSweepRows) + 1);
+    double* Dbuf = cv.take<double>(chol_scratch_doubles(cols));
+    const bool want_loss = H_undamped && loss_out;
+
+    { Launch l(K_DYN_AUX, stream); iota_kernel<<<cdiv(cols, 256), 256, 0, stream>>>(obuf[0], cols); }
+    const int32_t* ocur = obuf[0];           // original column index of every current position
+    // current state: the m columns still to do, their matrix (upper triangle valid) and their weights
+    const double* Acur = Hinv;
+    int64_t lda = cols;
+    const double* Wcur = nullptr;            // round 0 reads the float32 weights
+    int64_t ldc = 0;
+    int m = cols, done = 0, cur = 0;
+    while (m > 0) {
+        const int b = block < m ? block : m;
+        { Launch l(K_DYN_AUX, stream); extract_diag_ld_kernel<<<cdiv(m, 256), 256, 0, stream>>>(Acur, lda, m, diag); }
+        if (mode != PTQ_SCORE_NONE) {
+            Launch l(K_SCORE_PARTIAL, stream);
+            if (Wcur)
+                score_partial_kernel<double><<<dim3(cdiv(m, 128), chunks), 128, 0, stream>>>(Wcur, rows, m, ldc, scale, zero,
+                                                                                         bits, mode, partial);
+            else
+                score_partial_kernel<float><<<dim3(cdiv(m, 128), chunks), 128, 0, stream>>>(W, rows, m, ldw, scale, zero,
+                                                                                        bits, mode, partial);
+        }
+        { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(m, 128), 128, 0, stream>>>(partial, chunks, m, diag, mode, S, status); }
+        { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(m, kRankCols), 256, 0, stream>>>(S, m, ascending, ordr, ocur); }
+        double* An = Abuf[cur];
+        double* Wn = Wbuf[cur];
+        int32_t* onew = obuf[cur ^ 1];
+        {
+            Launch l(K_DYN_GATHER, stream);
+            const int gy = m < 4096 ? m : 4096, gr = rows < 4096 ? rows : 4096;
+            gather_upper_kernel<<<dim3(grid_x_for(m, 256), gy), 256, 0, stream>>>(Acur, lda, ordr, m, An);
+            if (Wcur)
+                gather_cols_kernel<double><<<dim3(grid_x_for(m, 256), gr), 256, 0, stream>>>(Wcur, ldc, rows, m, ordr, Wn);
+            else
+                gather_cols_kernel<float><<<dim3(grid_x_for(m, 256), gr), 256, 0, stream>>>(W, ldw, rows, m, ordr, Wn);
+            gather_index_kernel<<<cdiv(m, 256), 256, 0, stream>>>(ocur, ordr, m, b, onew, order_out + done);
+        }
+        int st = cholesky_upper(An, m, nullptr, Dbuf, bar, status, stream, b < m ? b / kNB : 0);
+        if (st) return st;
+        st = sweep_launch(Wn, An, E, codes_p, scale, zero, rows, b, bits, sweep_flags, status, stream, m);
+        if (st) return st;
+        if (b < m) {
+            // Eq. 11 for the columns still to come, all b columns at once: Wn[:, b:] -= E[:, :b] U[:b, b:]
+            GemmParams g = gemm_defaults();
+            g.A = E; g.lda = m; g.a_trans = 0;
+            g.B = An + b; g.ldb = m; g.b_trans = 0;
+            g.C = Wn + b; g.ldc = m;
+            g.M = rows; g.N = m - b; g.K = b;
+            g.alpha = -1.0; g.beta = 1.0;
+            st = launch_dgemm(K_DGEMM_DYN, g, 1, stream);
+            if (st) return st;
+        }
+        {
+            Launch l(K_DYN_AUX, stream);
+            const int gr = rows < 4096 ? rows : 4096;
+            emit_block_kernel<<<dim3(grid_x_for(b, 256), gr), 256, 0, stream>>>(codes_p, m, onew, b, W, rows, cols, ldw,
+                                                                            scale, zero, codes, What,
+                                                                            want_loss ? dW : nullptr);
+        }
+        Acur = An + (size_t)b * m + b; lda = m;
+        Wcur = Wn + b; ldc = m;
+        // what is left of the gathered arrays is the next round's state; the next round gathers into the other buffers
+        ocur = onew + b;
+        done += b;
+        m -= b;
+        cur ^= 1;
+    }
+    if (want_loss) {
+        GemmParams g = gemm_defaults();
+        g.kend_mode = 1; g.sym_double = 1;
+        g.A = dW; g.lda = cols; g.a_trans = 0;
+        g.B = H_undamped; g.ldb = cols; g.b_trans = 0;
+        g.M = rows; g.N = cols; g.K = cols;
+        g.D = dW; g.ldd = cols; g.partials = partials;
+        g.ksplit = loss_ksplit(rows, cols);
+        dim3 grid;
+        const int st = launch_dgemm(K_DGEMM_LOSS, g, 1, stream, 64, &grid);
+        if (st) return st;
+        { Launch l(K_SUM_PARTIALS, stream); sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y * grid.z), 0.5, loss_out); }
+    }
+    return launch_status();
 }
 
 int ptq_sort_scores(const double* S, int cols, int ascending, int32_t* perm, void* stream_) {

@@ -182,7 +182,13 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
             const bool ok = d0 > 0.0 && d0 < 1.0e300;
             bad = (!ok && bad < 0) ? p : bad;
             const double d = ok ? d0 : 1.0;
-            const double rs = rsqrt(d);
+            // 1 / sqrt(d): the hardware's approximation (about 20 bits) refined without a branch by
+            // y (1 + e / 2 + 3 e^2 / 8), e = 1 - d y^2, which leaves an error of order e^3, far below one ulp;
+            // the library routine is three times as long a chain
+            double y;
+            asm("rsqrt.approx.ftz.f64 %0, %1;" : "=d"(y) : "d"(d));
+            const double e = fma(-(y * y), d, 1.0);
+            const double rs = fma(y, e * fma(0.375, e, 0.5), y);
             const double inv = rs * rs;
             const double tx = x[p] * inv;
             x[p] *= rs;
@@ -458,7 +464,7 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int6
 
 __global__ void __launch_bounds__(kCholThreads, 1)
 chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __restrict__ Dbuf, int n, int64_t ld,
-                 int vec16, unsigned* bar, int32_t* status, long long spin_limit) {
+                 int vec16, unsigned* bar, int32_t* status, long long spin_limit, int nb_stop) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
     int* s_flag = reinterpret_cast<int*>(opnd + 2 * 2 * kNB * kCholLd);     // the strip panels alias opnd
@@ -569,11 +575,20 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         cp_async_wait<0>();
     };
 
+    // nb_stop < nb: a partial factorisation.  Only the first nb_stop block rows are factorised; their updates are applied
+    // to everything below, so that the upper triangle of A[64 nb_stop :, 64 nb_stop :] ends up holding the Schur
+    // complement of the leading block (what Eq. 12 leaves after that many columns).
+    const int nbs = nb_stop < nb ? nb_stop : nb;
+    const int steps = nbs < nb ? nbs : nb - 1;
     strip_phase(0);
-    for (int k = 0; k + 1 < nb; ++k) {
+    for (int k = 0; k < steps; ++k) {
         ++epoch;
         if (!grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) break;
         // Block row k is final; the updates of block rows < k have been applied everywhere.
+        if (k + 1 >= nbs) {                  // last factorised block row of a partial run: its update only
+            trailing_phase(k, k + 1, 0);
+            continue;
+        }
         const int next_items = strip_items(k + 1) > 0 ? strip_items(k + 1) : 1;
         // Look-ahead pays when giving up next_items CTAs lengthens the trailing phase by less than the strip phase and
         // the extra grid barrier it saves: compare rounds of tiles (about 4 us each) with and without, plus about 19 us.
@@ -616,7 +631,7 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
     // the diagonal factors move from the side buffer into A once nobody reads the original diagonal blocks any more
     ++epoch;
     if (grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) {
-        for (int b = blockIdx.x; b < nb; b += G)
+        for (int b = blockIdx.x; b < nbs; b += G)
             for (int idx = tid; idx < kNB * kNB; idx += kCholThreads) {
                 const int r = idx >> 6, c = idx & 63;
                 if (c >= r && b * kNB + c < n)
@@ -632,8 +647,12 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
 // Sec. 5 item 1 asks for.
 // `bar` is 2 x uint32 of device scratch, Dbuf holds chol_scratch_doubles(n) doubles (the diagonal factors on their way).
 inline size_t chol_scratch_doubles(int n) { return (size_t)((n + kNB - 1) / kNB) * kNB * kNB; }
+// nb_stop > 0: factorise the first nb_stop block rows of 64 only and leave the Schur complement of that leading block in
+// the upper triangle of the rest (Wm must be null then).
 inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* bar, int32_t* status,
-                          cudaStream_t stream) {
+                          cudaStream_t stream, int nb_stop = 0) {
+    if (nb_stop > 0 && Wm != nullptr) return PTQ_ERR_INVALID_ARG;
+    if (nb_stop <= 0) nb_stop = (n + kNB - 1) / kNB;
     DeviceState* dev = nullptr;
     int st = current_device_state(&dev);
     if (st) return st;
@@ -652,7 +671,7 @@ inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* 
     int64_t ld = n;
     int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;
     long long spin_limit = kSpinLimitCycles;
-    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status, &spin_limit};
+    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status, &spin_limit, &nb_stop};
     Launch l(K_CHOL_COOP, stream);
     if (cudaLaunchCooperativeKernel((const void*)chol_coop_kernel, dim3(grid), dim3(kCholThreads), args,
                                     kCholSmemBytes, stream) != cudaSuccess) {

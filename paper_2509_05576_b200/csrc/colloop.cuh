@@ -83,7 +83,8 @@ struct SweepParams {
     uint8_t* codes_p;       // [rows x n] codes in permuted order
     const float* scale;
     const float* zero;
-    int rows, n, bits, vec16;
+    int rows, n, bits, vec16;     // n: columns to sweep (the first n of each row)
+    int64_t ld;                   // row stride of Wp, U, E and codes_p (>= n)
     unsigned* flags;        // [groups] published 8-column pieces of E per group, then [1] abort word; zero at launch
     int32_t* status;
     long long spin_limit;   // SM clock cycles after which a wait on another CTA gives up
@@ -182,6 +183,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int rows = prm.rows, n = prm.n;
+    const int64_t ld = prm.ld;
     const int nb = (n + kNB - 1) / kNB;
     const int groups = (rows + kSweepRows - 1) / kSweepRows;
     const int G = gridDim.x;
@@ -208,7 +210,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
         for (int idx = tid; idx < kNB * kNB; idx += kSweepThreads) {
             const int r = idx >> 6, c = idx & 63;
             double v = (r == c) ? 1.0 : 0.0;
-            if (r < kb && c < kb && c >= r) v = __ldcg(prm.U + (int64_t)(p0 + r) * n + p0 + c);
+            if (r < kb && c < kb && c >= r) v = __ldcg(prm.U + (int64_t)(p0 + r) * ld + p0 + c);
             Us[r * kSweepLd + c] = v;
         }
         __syncthreads();
@@ -244,14 +246,14 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
             const bool next2_mine = cpg >= 4 && b + 2 < nb && ((b + 2) % cpg) == ci;
             if (next2_mine) {
                 __syncthreads();
-                sweep_load_tile(Bb, kSweepLd, prm.U, n, p0, p0 + 2 * kNB, kNB, kNB, n, n, prm.vec16);
+                sweep_load_tile(Bb, kSweepLd, prm.U, ld, p0, p0 + 2 * kNB, kNB, kNB, n, n, prm.vec16);
                 cp_async_commit();
                 load_diag(b + 2);            // nothing of it depends on E: out of the way two blocks early
             }
             if (next_mine) {
                 // block b + 1 is quantized here next: what does not depend on E[:, b] is fetched before waiting for it
                 __syncthreads();
-                sweep_load_tile(Bb, kSweepLd, prm.U, n, p0, p0 + kNB, kNB, kNB, n, n, prm.vec16);
+                sweep_load_tile(Bb, kSweepLd, prm.U, ld, p0, p0 + kNB, kNB, kNB, n, n, prm.vec16);
                 cp_async_commit();
                 if (!ahead) load_diag(b + 1);
             }
@@ -265,7 +267,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const int r = r0 + 8 * a + lq, c = p0 + 8 * warp + 2 * lr + e;
-                            blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
+                            blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * ld + c) : 0.0;
                         }
                 }
                 __syncthreads();
@@ -304,7 +306,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                         // (the warps to the right are already updating): the owner of the next block folds them into its
                         // block while the rest of this block is still being quantized.
                         if (live) {
-                            double* dst = prm.E + (int64_t)row * n + p0 + 8 * m;
+                            double* dst = prm.E + (int64_t)row * ld + p0 + 8 * m;
 #pragma unroll
                             for (int c = 0; c < 8; ++c) {
                                 v[c] *= rdiag[8 * m + c];
@@ -356,7 +358,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                 __syncthreads();
                 for (int idx = tid; idx < kSweepRows * kNB; idx += kSweepThreads) {
                     const int r = idx >> 6, c = idx & 63;
-                    if (r0 + r < rows && c < kb) prm.codes_p[(int64_t)(r0 + r) * n + p0 + c] = Cs[r * (kNB + 4) + c];
+                    if (r0 + r < rows && c < kb) prm.codes_p[(int64_t)(r0 + r) * ld + p0 + c] = Cs[r * (kNB + 4) + c];
                 }
                 prepared = false;
             } else if (!next_mine && !next2_mine) {
@@ -386,12 +388,12 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const int r = r0 + 8 * a + lq, c = c0 + 8 * warp + 2 * lr + e;
-                            blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * n + c) : 0.0;
+                            blk[a][e] = (r < rows && c < n) ? __ldcg(prm.Wp + (int64_t)r * ld + c) : 0.0;
                         }
                 }
                 // whatever of E[:, b] is out already comes in one go through shared memory (an owner that arrives late
                 // would otherwise pay one L2 round trip per piece); the pieces still missing there are polled below
-                sweep_load_tile(Ea, kSweepLd, prm.E, n, r0, p0, kSweepRows, kNB, rows, n, prm.vec16);
+                sweep_load_tile(Ea, kSweepLd, prm.E, ld, r0, p0, kSweepRows, kNB, rows, n, prm.vec16);
                 cp_async_commit();
                 cp_async_wait<0>();
                 __syncthreads();             // U[b, b + 1] (or U[b, b + 2]) is in Bb, the snapshot of E[:, b] in Ea
@@ -427,7 +429,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                                 for (int a = 0; a < 4; ++a) {
                                     const int r = r0 + 8 * a + lq;
                                     const double x =
-                                        r < rows ? ld_relaxed_f64(prm.E + (int64_t)r * n + p0 + 8 * m + 4 * s4 + lr) : 0.0;
+                                        r < rows ? ld_relaxed_f64(prm.E + (int64_t)r * ld + p0 + 8 * m + 4 * s4 + lr) : 0.0;
                                     af[m & 1][s4][a] = x;
                                     have = have && x == x;
                                 }
@@ -469,13 +471,13 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
             for (int e = e_lo; e <= b; ++e) {
                 // operand A: E[r0 .. r0+31][64 e .. 64 e + 63]
                 __syncthreads();
-                sweep_load_tile(Ea, kSweepLd, prm.E, n, r0, e * kNB, kSweepRows, kNB, rows, n, prm.vec16);
+                sweep_load_tile(Ea, kSweepLd, prm.E, ld, r0, e * kNB, kSweepRows, kNB, rows, n, prm.vec16);
                 int stage = 0;
-                sweep_load_tile(Bb, kSweepLd, prm.U, n, e * kNB, b_first * kNB, kNB, kNB, n, n, prm.vec16);
+                sweep_load_tile(Bb, kSweepLd, prm.U, ld, e * kNB, b_first * kNB, kNB, kNB, n, n, prm.vec16);
                 cp_async_commit();
                 for (int bp = b_first; bp < nb; bp += cpg) {
                     if (bp + cpg < nb)
-                        sweep_load_tile(Bb + (stage ^ 1) * kNB * kSweepLd, kSweepLd, prm.U, n, e * kNB,
+                        sweep_load_tile(Bb + (stage ^ 1) * kNB * kSweepLd, kSweepLd, prm.U, ld, e * kNB,
                                         (bp + cpg) * kNB, kNB, kNB, n, n, prm.vec16);
                     cp_async_commit();
                     // old values of the tile first (their latency hides behind the MMAs)
@@ -490,7 +492,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
                             const int c = j0 + wn0 + q * 8 + 2 * lr;
                             keep[a][q][0] = r < rows && c < n;
                             keep[a][q][1] = r < rows && c + 1 < n;
-                            const double* src = prm.Wp + (int64_t)r * n + c;
+                            const double* src = prm.Wp + (int64_t)r * ld + c;
                             if (prm.vec16 && keep[a][q][0]) {
                                 const double2 v = __ldcg(reinterpret_cast<const double2*>(src));
                                 old[a][q][0] = v.x;
@@ -523,7 +525,7 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 #pragma unroll
                         for (int q = 0; q < 2; ++q) {
                             const int c = j0 + wn0 + q * 8 + 2 * lr;
-                            double* dst = prm.Wp + (int64_t)r * n + c;
+                            double* dst = prm.Wp + (int64_t)r * ld + c;
                             const double v0 = old[a][q][0] - acc[a][q][0], v1 = old[a][q][1] - acc[a][q][1];
                             if (prm.vec16 && keep[a][q][0]) {
                                 __stcg(reinterpret_cast<double2*>(dst), make_double2(v0, v1));
@@ -544,8 +546,12 @@ __global__ void __launch_bounds__(kSweepThreads, 1) sweep_coop_kernel(SweepParam
 }
 
 // Launches the sweep: one CTA per SM, cooperative so that every CTA a waiting CTA depends on is resident.
+// n columns are swept; ld (0: n) is the row stride of Wp, U, E and codes_p, so that the first n columns of wider
+// arrays can be swept (the rows of U beyond column n are then applied by the caller).
 inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p, const float* scale, const float* zero,
-                        int rows, int n, int bits, unsigned* flags, int32_t* status, cudaStream_t stream) {
+                        int rows, int n, int bits, unsigned* flags, int32_t* status, cudaStream_t stream,
+                        int64_t ld = 0) {
+    if (ld == 0) ld = n;
     DeviceState* dev = nullptr;
     int st = current_device_state(&dev);
     if (st) return st;
@@ -563,11 +569,11 @@ inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p
     const int groups = cdiv(rows, kSweepRows);
     if (cudaMemsetAsync(flags, 0, ((size_t)groups + 1) * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     // every byte 0xFF is a NaN: "not published yet" for the owner of the next block, which polls the values themselves
-    if (cudaMemsetAsync(E, 0xFF, (size_t)rows * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
+    if (cudaMemsetAsync(E, 0xFF, (size_t)rows * ld * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     SweepParams prm;
     prm.Wp = Wp; prm.U = U; prm.E = E; prm.codes_p = codes_p; prm.scale = scale; prm.zero = zero;
-    prm.rows = rows; prm.n = n; prm.bits = bits;
-    prm.vec16 = ((n & 1) == 0 && aligned16(Wp) && aligned16(U) && aligned16(E)) ? 1 : 0;
+    prm.rows = rows; prm.n = n; prm.bits = bits; prm.ld = ld;
+    prm.vec16 = ((n & 1) == 0 && (ld & 1) == 0 && aligned16(Wp) && aligned16(U) && aligned16(E)) ? 1 : 0;
     prm.flags = flags; prm.status = status; prm.spin_limit = kSpinLimitCycles;
     void* args[] = {&prm};
     Launch l(K_SWEEP_COOP, stream);

@@ -136,7 +136,8 @@ enum KernelId {
     K_GRAM_SPLIT = 0, K_GRAM_I8, K_GRAM_FINISH, K_CONVERT_F64, K_DGEMM_GRAM, K_LAMBDA, K_DAMP_COPY, K_CHOL_COOP,
     K_DGEMM_LAUUM, K_EXTRACT_DIAG, K_MINMAX_GRID, K_SCORE_PARTIAL,
     K_SCORE_FINAL, K_RANK_SORT, K_PERM_CHECK, K_GATHER_SYM, K_GATHER_W, K_SWEEP_COOP, K_FINALIZE,
-    K_DGEMM_LOSS, K_SUM_PARTIALS, K_SELFTEST, K_FP64_PROBE, K_COUNT
+    K_DGEMM_LOSS, K_SUM_PARTIALS, K_SELFTEST, K_FP64_PROBE, K_DYN_AUX, K_DYN_GATHER,
+    K_DGEMM_DYN, K_COUNT
 };
 
 inline const char* kernel_name(int id) {
@@ -144,7 +145,8 @@ inline const char* kernel_name(int id) {
         "gram_split", "gram_i8_tcgen05", "gram_finish", "convert_f64", "dgemm_gram_f64", "lambda", "damp_copy", "chol_coop",
         "dgemm_lauum", "extract_diag",
         "minmax_grid", "score_partial", "score_final", "rank_sort", "perm_check", "gather_sym", "gather_w",
-        "sweep_coop", "finalize", "dgemm_loss", "sum_partials", "selftest_wait", "fp64_probe"};
+        "sweep_coop", "finalize", "dgemm_loss", "sum_partials", "selftest_wait", "fp64_probe", "dyn_aux", "dyn_gather",
+        "dgemm_dyn"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

@@ -56,8 +56,10 @@ __global__ void __launch_bounds__(256) minmax_grid_kernel(const float* __restric
 
 constexpr int kScoreRowChunk = 64;
 
-// partial[ch][j] = sum over the rows of chunk ch (ascending) of the score numerator of w_ij.
-__global__ void __launch_bounds__(128) score_partial_kernel(const float* __restrict__ W, int rows, int cols,
+// partial[ch][j] = sum over the rows of chunk ch (ascending) of the score numerator of w_ij.  T = float for the original
+// weights, double for the compensated weights that dynamic re-ranking scores.
+template <typename T>
+__global__ void __launch_bounds__(128) score_partial_kernel(const T* __restrict__ W, int rows, int cols,
                                                              int64_t ldw, const float* __restrict__ scale,
                                                              const float* __restrict__ zero, int bits, int mode,
                                                              double* __restrict__ partial) {
@@ -108,22 +110,29 @@ __device__ __forceinline__ unsigned long long sortable_key(double x) {
 // (ascending != 0: S_k < S_j instead, the "asc" keys of Sec. 4.1; equal scores keep the lower index first either way).
 // 32 columns j per CTA; the eight lanes that share a column each count a strided eighth of the keys.
 constexpr int kRankCols = 32;
+// tie != nullptr: equal scores are ordered by tie[] (distinct values) instead of by position.
 __global__ void __launch_bounds__(256) rank_sort_kernel(const double* __restrict__ S, int cols, int ascending,
-                                                         int32_t* __restrict__ perm) {
+                                                         int32_t* __restrict__ perm,
+                                                         const int32_t* __restrict__ tie = nullptr) {
     __shared__ unsigned long long keys[1024];
+    __shared__ int32_t ties[1024];
     const int j = blockIdx.x * kRankCols + (threadIdx.x >> 3);
     const int part = threadIdx.x & 7;
     // ascending order is descending order of the complemented keys
     const unsigned long long flip = ascending ? ~0ull : 0ull;
     const unsigned long long kj = j < cols ? (sortable_key(S[j]) ^ flip) : 0ull;
+    const int tj = (tie != nullptr && j < cols) ? tie[j] : j;
     int rank = 0;
     for (int t0 = 0; t0 < cols; t0 += 1024) {
-        for (int t = threadIdx.x; t < 1024; t += 256) keys[t] = t0 + t < cols ? (sortable_key(S[t0 + t]) ^ flip) : 0ull;
+        for (int t = threadIdx.x; t < 1024; t += 256) {
+            keys[t] = t0 + t < cols ? (sortable_key(S[t0 + t]) ^ flip) : 0ull;
+            ties[t] = (tie != nullptr && t0 + t < cols) ? tie[t0 + t] : t0 + t;
+        }
         __syncthreads();
         const int lim = min(1024, cols - t0);
         for (int t = part; t < lim; t += 8) {
             const unsigned long long kk = keys[t];
-            rank += (kk > kj || (kk == kj && (t0 + t) < j)) ? 1 : 0;
+            rank += (kk > kj || (kk == kj && ties[t] < tj)) ? 1 : 0;
         }
         __syncthreads();
     }

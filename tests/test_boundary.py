@@ -38,7 +38,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_workspace_sizes(lib):
     from paper_2509_05576_b200 import ptq
-    for call in range(5):
+    for call in range(6):
         small = ptq.workspace_bytes(call, 64, 128, 1024)
         big = ptq.workspace_bytes(call, 256, 2304, 4096)
         assert 0 < small < big
@@ -96,6 +96,11 @@ def test_new_entry_points_check_their_arguments_on_the_host(lib):
     assert lib.ptq_sensitivity_order(*args, 5, fake, fake, fake, 1 << 20, fake, None) == ptq.ERR_INVALID_ARG
     assert lib.ptq_sensitivity_order(*args, 32, fake, fake, fake, 1 << 20, fake, None) == ptq.ERR_INVALID_ARG
     assert lib.ptq_sensitivity_order(*args, ptq.SCORE_W | ptq.SCORE_ASCENDING, fake, fake, None, 0, fake, None) == ptq.ERR_WORKSPACE
+    # dynamic re-ranking: rounds end on the 64-column block grid
+    dyn = (fake, 8, 200, 200, fake, fake, fake, 4, 0)
+    assert lib.ptq_quantize_layer_dynamic(*dyn, 100, fake, None, fake, None, None, fake, 1 << 40, fake, None) == ptq.ERR_UNSUPPORTED
+    assert lib.ptq_quantize_layer_dynamic(*dyn, 0, fake, None, fake, None, None, fake, 1 << 40, fake, None) == ptq.ERR_INVALID_ARG
+    assert lib.ptq_quantize_layer_dynamic(*dyn, 64, fake, None, fake, None, None, fake, 64, fake, None) == ptq.ERR_WORKSPACE
     # sizes beyond what the launch grid can index are refused, not launched
     assert lib.ptq_quantize_layer(fake, 70000, 8, 8, fake, fake, fake, fake, 4, fake, None, None, None, fake, 1 << 40,
                                   fake, None) == ptq.ERR_UNSUPPORTED
