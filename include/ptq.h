@@ -71,7 +71,8 @@ typedef enum {
     PTQ_CALL_SENSITIVITY_ORDER = 2,
     PTQ_CALL_QUANTIZE_LAYER = 3,
     PTQ_CALL_HESSIAN_ACCUMULATE_F64 = 4,
-    PTQ_CALL_QUANTIZE_LAYER_DYNAMIC = 5
+    PTQ_CALL_QUANTIZE_LAYER_DYNAMIC = 5,
+    PTQ_CALL_QUANTIZE_LAYER_PER_ROW = 6
 } ptq_call_id;
 
 /* Minimum workspace, in bytes, for one call with these sizes (host function, no CUDA calls). */
@@ -195,6 +196,21 @@ int ptq_quantize_layer(const float *W, int rows, int cols, int64_t ldw, const do
 int ptq_quantize_layer_dynamic(const float *W, int rows, int cols, int64_t ldw, const double *Hinv, const float *scale,
                                const float *zero, int bits, int score_mode, int block, uint8_t *codes, float *What,
                                int32_t *order_out, const double *H_undamped, double *loss_out, void *ws,
+                               size_t ws_bytes, int32_t *status, void *stream);
+
+/*
+ * The non-parallel arm of the paper's ablation (Sec. 4.2, the paragraph on the per-row inverse Hessians; Table 3's rows
+ * without the parallel tick): every row ranks its own weights by their sensitivities (the keys of
+ * ptq_sensitivity_order applied to that single row, Sec. 4.1) and is quantized in that order against its own copy of
+ * the inverse Hessian -- what the shared-inverse-Hessian method avoids.  Cost rows * cols^3 / 3 and one cols x cols
+ * matrix per row in flight, so only narrow layers are taken: cols <= 128 (PTQ_ERR_UNSUPPORTED beyond).
+ *   perm_rows [rows x cols] int32, out: the order each row used
+ *   other arguments as for ptq_quantize_layer; the diagonal of Hinv is read from Hinv itself
+ * Workspace: ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER_PER_ROW, rows, cols, 0).
+ */
+int ptq_quantize_layer_per_row(const float *W, int rows, int cols, int64_t ldw, const double *Hinv, const float *scale,
+                               const float *zero, int bits, int score_mode, uint8_t *codes, float *What,
+                               int32_t *perm_rows, const double *H_undamped, double *loss_out, void *ws,
                                size_t ws_bytes, int32_t *status, void *stream);
 
 /*

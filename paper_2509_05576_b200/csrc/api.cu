@@ -6,6 +6,7 @@
 #include "colloop.cuh"
 #include "gram.cuh"
 #include "dynamic.cuh"
+#include "perrow.cuh"
 
 using namespace ptq;
 
@@ -216,6 +217,10 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
             add(((size_t)cdiv(rows, kSweepRows) + 1) * sizeof(unsigned));   // per-row-group progress counters of the sweep
             add(chol_scratch_doubles(cols) * sizeof(double));
+            break;
+        case PTQ_CALL_QUANTIZE_LAYER_PER_ROW:
+            if (rows < 1) return 0;
+            add((size_t)rows * sizeof(double));             // per-row losses
             break;
         case PTQ_CALL_QUANTIZE_LAYER_DYNAMIC:
             if (rows < 1) return 0;
@@ -472,6 +477,44 @@ int ptq_quantize_layer_dynamic(const float* W, int rows, int cols, int64_t ldw, 
         const int st = launch_dgemm(K_DGEMM_LOSS, g, 1, stream, 64, &grid);
         if (st) return st;
         { Launch l(K_SUM_PARTIALS, stream); sum_partials_kernel<<<1, 256, 0, stream>>>(partials, (int)(grid.x * grid.y * grid.z), 0.5, loss_out); }
+    }
+    return launch_status();
+}
+
+int ptq_quantize_layer_per_row(const float* W, int rows, int cols, int64_t ldw, const double* Hinv, const float* scale,
+                               const float* zero, int bits, int score_mode, uint8_t* codes, float* What,
+                               int32_t* perm_rows, const double* H_undamped, double* loss_out, void* ws,
+                               size_t ws_bytes, int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!W || !Hinv || !scale || !zero || !codes || !perm_rows || rows < 1 || cols < 1 || ldw < cols || bits < 2 ||
+        bits > 8)
+        return PTQ_ERR_INVALID_ARG;
+    if (score_mode & ~(PTQ_SCORE_ASCENDING | 7)) return PTQ_ERR_INVALID_ARG;
+    const int mode = score_mode & ~PTQ_SCORE_ASCENDING, ascending = (score_mode & PTQ_SCORE_ASCENDING) ? 1 : 0;
+    if (mode < PTQ_SCORE_QERR || mode > PTQ_SCORE_NONE) return PTQ_ERR_INVALID_ARG;
+    if (cols > kPerRowMaxCols) return PTQ_ERR_UNSUPPORTED;       // one private inverse Hessian per CTA, in shared memory
+    if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_QUANTIZE_LAYER_PER_ROW, rows, cols, 0)) return PTQ_ERR_WORKSPACE;
+    if (!aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    DeviceState* dev = nullptr;
+    int st = current_device_state(&dev);
+    if (st) return st;
+    st = ensure_smem_attr(dev, SA_SMALL, [] {
+        return cudaFuncSetAttribute(per_row_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)per_row_smem_bytes(kPerRowMaxCols));
+    });
+    if (st) return st;
+    Carver cv(ws);
+    double* row_loss = cv.take<double>(rows);
+    const bool want_loss = H_undamped && loss_out;
+    {
+        Launch l(K_PER_ROW, stream);
+        per_row_kernel<<<rows, kPerRowThreads, per_row_smem_bytes(cols), stream>>>(
+            W, rows, cols, ldw, Hinv, scale, zero, bits, mode, ascending, codes, What, perm_rows,
+            want_loss ? H_undamped : nullptr, want_loss ? row_loss : nullptr, status);
+    }
+    if (want_loss) {
+        Launch l(K_SUM_PARTIALS, stream);
+        sum_partials_kernel<<<1, 256, 0, stream>>>(row_loss, rows, 1.0, loss_out);
     }
     return launch_status();
 }

@@ -23,10 +23,11 @@ SCORE_QERR, SCORE_PRUNE, SCORE_ERR, SCORE_W, SCORE_NONE = 0, 1, 2, 3, 4
 SCORE_ASCENDING = 16          # added to a score mode: sort by S ascending
 CALL_HESSIAN_ACCUMULATE, CALL_PREPARE_HINV, CALL_SENSITIVITY_ORDER, CALL_QUANTIZE_LAYER, CALL_HESSIAN_ACCUMULATE_F64 = range(5)
 CALL_QUANTIZE_LAYER_DYNAMIC = 5
+CALL_QUANTIZE_LAYER_PER_ROW = 6
 
 EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_conv", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
            "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_sensitivity_order_static", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
-           "ptq_sort_scores", "ptq_quantize_layer_dynamic", "ptq_selftest_wait_timeout", "ptq_fp64_probe",
+           "ptq_sort_scores", "ptq_quantize_layer_dynamic", "ptq_quantize_layer_per_row", "ptq_selftest_wait_timeout", "ptq_fp64_probe",
            "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
 
 
@@ -66,6 +67,8 @@ def lib():
         L.ptq_quantize_layer.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, vp, c_int, vp, vp, vp, vp, vp,
                                          c_size_t, vp, vp]
         L.ptq_sort_scores.argtypes = [vp, c_int, c_int, vp, vp]
+        L.ptq_quantize_layer_per_row.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, vp, vp,
+                                                 vp, c_size_t, vp, vp]
         L.ptq_quantize_layer_dynamic.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, c_int, vp, vp,
                                                  vp, vp, vp, vp, c_size_t, vp, vp]
         L.ptq_selftest_wait_timeout.argtypes = [c_int, ctypes.c_longlong, vp, c_size_t, vp, vp]
@@ -284,6 +287,19 @@ def quantize_layer_dynamic(W, Hinv, scale, zero, bits, score_mode, block, codes,
                                             int(bits), int(score_mode), int(block), _ptr(codes), _ptr(What),
                                             _ptr(order_out), _ptr(H_undamped), _ptr(loss_out), _ptr(buf), buf.numel(),
                                             _ptr(status), _stream(stream)), "ptq_quantize_layer_dynamic")
+
+
+def quantize_layer_per_row(W, Hinv, scale, zero, bits, score_mode, codes, What, perm_rows, H_undamped, loss_out, ws,
+                           status, stream=None):
+    """The non-parallel arm (Sec. 4.2): every row in its own order against its own inverse Hessian; cols <= 128."""
+    _dev(W, torch.float32, "W"); _dev(Hinv, torch.float64, "Hinv"); _dev(codes, torch.uint8, "codes")
+    _dev(perm_rows, torch.int32, "perm_rows")
+    rows, cols = W.shape
+    buf = ws.get(workspace_bytes(CALL_QUANTIZE_LAYER_PER_ROW, rows, cols, 0))
+    _check(lib().ptq_quantize_layer_per_row(_ptr(W), rows, cols, _rowmajor(W, "W"), _ptr(Hinv), _ptr(scale), _ptr(zero),
+                                            int(bits), int(score_mode), _ptr(codes), _ptr(What), _ptr(perm_rows),
+                                            _ptr(H_undamped), _ptr(loss_out), _ptr(buf), buf.numel(), _ptr(status),
+                                            _stream(stream)), "ptq_quantize_layer_per_row")
 
 
 class LayerBuffers:
