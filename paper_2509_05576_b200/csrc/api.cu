@@ -61,8 +61,8 @@ int order_launch(const float* W, int rows, int cols, int64_t ldw, const double* 
     if (chunks > 65535) return PTQ_ERR_UNSUPPORTED;
     if (mode != PTQ_SCORE_NONE) {
         Launch l(K_SCORE_PARTIAL, stream);
-        score_partial_kernel<float><<<dim3(cdiv(cols, 128), chunks), 128, 0, stream>>>(W, rows, cols, ldw, scale, zero,
-                                                                                     bits, mode, partial);
+        score_partial_kernel<float><<<dim3(cdiv(cols, kScoreCols), chunks), 256, 0, stream>>>(W, rows, cols, ldw, scale,
+                                                                                            zero, bits, mode, partial);
     }
     { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(cols, 128), 128, 0, stream>>>(partial, chunks, cols, Hinv_diag, mode, S, status); }
     { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(cols, kRankCols), 256, 0, stream>>>(S, cols, ascending, perm); }
@@ -414,11 +414,11 @@ int ptq_quantize_layer_dynamic(const float* W, int rows, int cols, int64_t ldw, 
         if (mode != PTQ_SCORE_NONE) {
             Launch l(K_SCORE_PARTIAL, stream);
             if (Wcur)
-                score_partial_kernel<double><<<dim3(cdiv(m, 128), chunks), 128, 0, stream>>>(Wcur, rows, m, ldc, scale, zero,
-                                                                                         bits, mode, partial);
+                score_partial_kernel<double><<<dim3(cdiv(m, kScoreCols), chunks), 256, 0, stream>>>(Wcur, rows, m, ldc, scale,
+                                                                                                zero, bits, mode, partial);
             else
-                score_partial_kernel<float><<<dim3(cdiv(m, 128), chunks), 128, 0, stream>>>(W, rows, m, ldw, scale, zero,
-                                                                                        bits, mode, partial);
+                score_partial_kernel<float><<<dim3(cdiv(m, kScoreCols), chunks), 256, 0, stream>>>(W, rows, m, ldw, scale,
+                                                                                               zero, bits, mode, partial);
         }
         { Launch l(K_SCORE_FINAL, stream); score_final_kernel<<<cdiv(m, 128), 128, 0, stream>>>(partial, chunks, m, diag, mode, S, status); }
         { Launch l(K_RANK_SORT, stream); rank_sort_kernel<<<cdiv(m, kRankCols), 256, 0, stream>>>(S, m, ascending, ordr, ocur); }

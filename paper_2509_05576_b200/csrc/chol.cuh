@@ -138,32 +138,68 @@ __device__ __forceinline__ void chol_load_block(double* dst, const double* __res
 // Strip factorisation: the 64 x 128 strip [diagonal block | 64 panel columns] is held in registers as 8 x 8
 // MMA accumulator fragments (warp w owns strip columns 16 w .. 16 w + 15, all 64 rows).  Pivots are taken eight
 // at a time.  For pivot block b:
-//   1. every warp publishes its piece of rows 8 b .. 8 b + 7 (the row panel R) to shared memory;
-//   2. four warps factorise the 8 x 8 diagonal mini-block M = U_M^T U_M (redundantly, all of M in every lane)
-//      and carry the identity along to obtain W = U_M^-T;
-//   3. the new rows U[8 b .. 8 b + 7][:] = W R come from two MMAs per fragment;
-//   4. they are published and subtracted from the rows below, A[i][c] -= U[p][i] U[p][c], again by MMA.
-// Three block-wide barriers per eight pivots; the only serial chain is the eight reciprocal square roots of step 2.
+//   1. warp 0 factorises the 8 x 8 diagonal mini-block M = U_M^T U_M (all of M in every lane, so the serial chain of
+//      eight pivots has no data exchange in it) and carries the identity along to obtain W = U_M^-T;
+//   2. the new rows U[8 b .. 8 b + 7][:] = W R come from two MMAs per fragment (R: the row panel, published before);
+//   3. they are published; every warp subtracts them from the rows of pivot block b + 1 FIRST and publishes those
+//      rows at once, so that warp 0 can start on the next mini-block,
+//   4. while the other warps subtract them from the rows further down, A[i][c] -= U[p][i] U[p][c], again by MMA.
+// Warp 0 owns the first 16 columns of the diagonal block, whose fragments below row 16 are never used: it has no
+// update work of its own in step 4 and is therefore the one that runs the chain.  Named barrier 1 hands the row panel
+// to warp 0 (the others only arrive), named barrier 2 hands W to everybody.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kStripLd = 132;                                            // row stride of the 8-row panels
-constexpr int kStripSmemDoubles = 2 * 8 * kStripLd + (kCholThreads / 32) * 64;
+constexpr int kStripSmemDoubles = 2 * 8 * kStripLd + 64;
 static_assert(kStripSmemDoubles <= 2 * 2 * kNB * kCholLd, "the strip panels alias the trailing-phase operand buffers");
+
+__device__ __forceinline__ void strip_bar_sync(int id) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(kCholThreads) : "memory");
+}
+__device__ __forceinline__ void strip_bar_arrive(int id) {
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(kCholThreads) : "memory");
+}
+
+// Rows of pivot block B of this warp's columns go to the row panel.
+template <int B>
+__device__ __forceinline__ void chol_strip_publish(const double (&acc)[8][2][2], double* Rbuf, int c0, int lq, int lr) {
+#pragma unroll
+    for (int cb = 0; cb < 2; ++cb)
+        *reinterpret_cast<double2*>(Rbuf + lq * kStripLd + c0 + 8 * cb + 2 * lr) =
+            make_double2(acc[B][cb][0], acc[B][cb][1]);
+}
+
+// acc[r] -= U[:, 8 r .. 8 r + 7]^T U[:, own columns] for the fragment rows R0 <= r < R1 (U: the eight rows in Ubuf).
+template <int R0, int R1>
+__device__ __forceinline__ void chol_strip_update(double (&acc)[8][2][2], const double* Ubuf, int warp, int c0, int lq,
+                                                  int lr) {
+    if constexpr (R0 < R1) {
+        double bf[2][2];
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+            bf[cb][0] = Ubuf[lr * kStripLd + c0 + 8 * cb + lq];
+            bf[cb][1] = Ubuf[(4 + lr) * kStripLd + c0 + 8 * cb + lq];
+        }
+#pragma unroll
+        for (int r = R0; r < R1; ++r) {
+            const double n0 = -Ubuf[lr * kStripLd + 8 * r + lq];
+            const double n1 = -Ubuf[(4 + lr) * kStripLd + 8 * r + lq];
+#pragma unroll
+            for (int cb = 0; cb < 2; ++cb) {
+                if (warp < 4 && 8 * r > c0 + 8 * cb + 7) continue;       // entirely below the diagonal: never used
+                dmma_884(acc[r][cb][0], acc[r][cb][1], n0, bf[cb][0]);
+                dmma_884(acc[r][cb][0], acc[r][cb][1], n1, bf[cb][1]);
+            }
+        }
+    }
+}
 
 template <int B>
 __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
                                                  int warp, int lane, int k0, bool reporter, int32_t* status) {
     const int lq = lane >> 2, lr = lane & 3;
     const int c0 = 16 * warp;
-    // 1. publish the row panel
-#pragma unroll
-    for (int cb = 0; cb < 2; ++cb)
-        *reinterpret_cast<double2*>(Rbuf + lq * kStripLd + c0 + 8 * cb + 2 * lr) =
-            make_double2(acc[B][cb][0], acc[B][cb][1]);
-    __syncthreads();
-    // 2. warps 0..3 (one per scheduler) each factorise M; every lane holds all of M, so the serial chain of
-    //    eight reciprocal square roots has no data exchange in it.  Lane j carries column j of the identity along,
-    //    which becomes column j of W = U_M^-T.
-    if (warp < 4) {
+    if (warp == 0) {
+        // 1. the mini-block; lane j carries column j of the identity along, which becomes column j of W = U_M^-T
         double m[8][8];
 #pragma unroll
         for (int p = 0; p < 8; ++p)
@@ -202,14 +238,16 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
         }
         if (lane < 8) {
 #pragma unroll
-            for (int p = 0; p < 8; ++p) Wbuf[warp * 64 + p * 8 + lane] = x[p];    // W[p][j] = (U_M^-T)[p][j]
+            for (int p = 0; p < 8; ++p) Wbuf[p * 8 + lane] = x[p];    // W[p][j] = (U_M^-T)[p][j]
         }
         if (bad >= 0 && reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + bad);
+    } else if constexpr (B > 0) {
+        // 4. (of the mini-block before) the rows further down, while warp 0 is in its chain
+        chol_strip_update<B + 1, 8>(acc, Ubuf, warp, c0, lq, lr);
     }
-    __syncthreads();
-    const double* wb = Wbuf + (warp & 3) * 64;
-    // 3. new rows = W R
-    const double a0 = wb[lq * 8 + lr], a1 = wb[lq * 8 + 4 + lr];
+    strip_bar_sync(2);       // W is there; nobody reads the previous new rows any more
+    // 2. new rows = W R
+    const double a0 = Wbuf[lq * 8 + lr], a1 = Wbuf[lq * 8 + 4 + lr];
 #pragma unroll
     for (int cb = 0; cb < 2; ++cb) {
         const double b0 = Rbuf[lr * kStripLd + c0 + 8 * cb + lq];
@@ -222,31 +260,19 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
         *reinterpret_cast<double2*>(Ubuf + lq * kStripLd + c0 + 8 * cb + 2 * lr) = make_double2(r0, r1);
     }
     __syncthreads();
-    // 4. rows below: acc[r] -= U[:, 8 r .. 8 r + 7]^T U[:, own columns]
+    // 3. the rows of the next pivot block first, and out they go
     if constexpr (B < 7) {
-        double bf[2][2];
-#pragma unroll
-        for (int cb = 0; cb < 2; ++cb) {
-            bf[cb][0] = Ubuf[lr * kStripLd + c0 + 8 * cb + lq];
-            bf[cb][1] = Ubuf[(4 + lr) * kStripLd + c0 + 8 * cb + lq];
-        }
-#pragma unroll
-        for (int r = B + 1; r < 8; ++r) {
-            const double n0 = -Ubuf[lr * kStripLd + 8 * r + lq];
-            const double n1 = -Ubuf[(4 + lr) * kStripLd + 8 * r + lq];
-#pragma unroll
-            for (int cb = 0; cb < 2; ++cb) {
-                if (warp < 4 && 8 * r > c0 + 8 * cb + 7) continue;       // entirely below the diagonal: never used
-                dmma_884(acc[r][cb][0], acc[r][cb][1], n0, bf[cb][0]);
-                dmma_884(acc[r][cb][0], acc[r][cb][1], n1, bf[cb][1]);
-            }
-        }
+        chol_strip_update<B + 1, B + 2>(acc, Ubuf, warp, c0, lq, lr);
+        chol_strip_publish<B + 1>(acc, Rbuf, c0, lq, lr);
+        if (warp == 0) strip_bar_sync(1); else strip_bar_arrive(1);
     }
 }
 template <int... Bs>
 __device__ __forceinline__ void chol_strip_blocks(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
                                                   int warp, int lane, int k0, bool reporter, int32_t* status,
                                                   std::integer_sequence<int, Bs...>) {
+    chol_strip_publish<0>(acc, Rbuf, 16 * warp, lane >> 2, lane & 3);
+    if (warp == 0) strip_bar_sync(1); else strip_bar_arrive(1);
     (chol_strip_block<Bs>(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, reporter, status), ...);
 }
 

@@ -56,33 +56,50 @@ __global__ void __launch_bounds__(256) minmax_grid_kernel(const float* __restric
 
 constexpr int kScoreRowChunk = 64;
 
-// partial[ch][j] = sum over the rows of chunk ch (ascending) of the score numerator of w_ij.  T = float for the original
-// weights, double for the compensated weights that dynamic re-ranking scores.
+// partial[ch][j] = sum over the rows of chunk ch of the score numerator of w_ij.  T = float for the original weights,
+// double for the compensated weights that dynamic re-ranking scores.
+// One CTA per 64-row chunk and 32 columns: thread (g, c) adds rows 8 g .. 8 g + 7 of column c in ascending order (eight
+// independent loads in flight), then the eight sub-sums of a column are added in ascending g: a fixed order, so the
+// result does not depend on the launch.
+constexpr int kScoreCols = 32;
 template <typename T>
-__global__ void __launch_bounds__(128) score_partial_kernel(const T* __restrict__ W, int rows, int cols,
+__global__ void __launch_bounds__(256) score_partial_kernel(const T* __restrict__ W, int rows, int cols,
                                                              int64_t ldw, const float* __restrict__ scale,
                                                              const float* __restrict__ zero, int bits, int mode,
                                                              double* __restrict__ partial) {
-    const int j = blockIdx.x * 128 + threadIdx.x;
+    __shared__ double sub[8][kScoreCols + 1];
+    const int c = threadIdx.x & (kScoreCols - 1), g = threadIdx.x / kScoreCols;
+    const int j = blockIdx.x * kScoreCols + c;
     const int ch = blockIdx.y;
-    if (j >= cols) return;
-    const int r0 = ch * kScoreRowChunk;
-    const int r1 = min(rows, r0 + kScoreRowChunk);
+    const int r0 = ch * kScoreRowChunk + g * (kScoreRowChunk / 8);
     const double maxq = (double)((1 << bits) - 1);
     const bool use_err = (mode == PTQ_SCORE_QERR || mode == PTQ_SCORE_ERR);
     double s = 0.0;
-    for (int i = r0; i < r1; ++i) {
-        const double w = (double)W[(int64_t)i * ldw + j];
-        if (use_err) {
-            const double sc = (double)scale[i], zp = (double)zero[i];
-            const double q = sc * (quant_code_d(w, sc, zp, maxq) - zp);
-            const double d = w - q;
-            s = fma(d, d, s);
-        } else {
-            s = fma(w, w, s);
+    if (j < cols) {
+        double w[kScoreRowChunk / 8];
+#pragma unroll
+        for (int k = 0; k < kScoreRowChunk / 8; ++k) w[k] = r0 + k < rows ? (double)W[(int64_t)(r0 + k) * ldw + j] : 0.0;
+#pragma unroll
+        for (int k = 0; k < kScoreRowChunk / 8; ++k) {
+            if (r0 + k >= rows) break;
+            if (use_err) {
+                const double sc = (double)scale[r0 + k], zp = (double)zero[r0 + k];
+                const double q = sc * (quant_code_d(w[k], sc, zp, maxq) - zp);
+                const double d = w[k] - q;
+                s = fma(d, d, s);
+            } else {
+                s = fma(w[k], w[k], s);
+            }
         }
     }
-    partial[(int64_t)ch * cols + j] = s;
+    sub[g][c] = s;
+    __syncthreads();
+    if (g == 0 && j < cols) {
+        double t = sub[0][c];
+#pragma unroll
+        for (int k = 1; k < 8; ++k) t += sub[k][c];
+        partial[(int64_t)ch * cols + j] = t;
+    }
 }
 
 // S_j = (sum of the chunk partials, ascending) / (2 [Hinv]_jj)  for the sensitivity modes.
