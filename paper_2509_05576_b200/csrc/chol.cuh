@@ -193,9 +193,34 @@ __device__ __forceinline__ void chol_strip_update(double (&acc)[8][2][2], const 
     }
 }
 
+// Look-ahead update of fragment row RB of this warp's strip columns with the block row above (see chol_strip):
+//     acc[RB] -= ua[:, 8 RB .. 8 RB + 7]^T bsrc[:, own 16 columns]        (ua, bsrc: 64 x 64 in shared memory)
+// Applied one fragment row at a time, just before the row is needed, by the warps that wait for warp 0's chain.
+template <int RB>
+__device__ __forceinline__ void chol_strip_lookahead(double (&acc)[8][2][2], const double* ua, const double* bsrc,
+                                                     bool is_diag, int sc0, int lq, int lr) {
+    double prod[2][2] = {{0.0, 0.0}, {0.0, 0.0}};
+#pragma unroll 4
+    for (int kk = 0; kk < kNB; kk += 4) {
+        const double af = ua[(kk + lr) * kCholLd + 8 * RB + lq];
+#pragma unroll
+        for (int cb = 0; cb < 2; ++cb) {
+            // fragments of the diagonal block that lie entirely below the diagonal are never used
+            if (is_diag && 8 * RB > sc0 + 8 * cb + 7) continue;
+            dmma_884(prod[cb][0], prod[cb][1], af, bsrc[(kk + lr) * kCholLd + 8 * cb + lq]);
+        }
+    }
+#pragma unroll
+    for (int cb = 0; cb < 2; ++cb) {
+        acc[RB][cb][0] -= prod[cb][0];
+        acc[RB][cb][1] -= prod[cb][1];
+    }
+}
+
 template <int B>
 __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
-                                                 int warp, int lane, int k0, bool reporter, int32_t* status) {
+                                                 int warp, int lane, int k0, bool reporter, int32_t* status,
+                                                 const double* ua, const double* bsrc) {
     const int lq = lane >> 2, lr = lane & 3;
     const int c0 = 16 * warp;
     if (warp == 0) {
@@ -241,9 +266,13 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
             for (int p = 0; p < 8; ++p) Wbuf[p * 8 + lane] = x[p];    // W[p][j] = (U_M^-T)[p][j]
         }
         if (bad >= 0 && reporter) report(status, PTQ_ERR_NOT_SPD, k0 + 8 * B + bad);
-    } else if constexpr (B > 0) {
-        // 4. (of the mini-block before) the rows further down, while warp 0 is in its chain
-        chol_strip_update<B + 1, 8>(acc, Ubuf, warp, c0, lq, lr);
+    } else {
+        // while warp 0 is in its chain: 4. (of the mini-block before) the rows further down, and the look-ahead update
+        // of the rows of the next pivot block, which are needed right after this mini-block
+        if constexpr (B > 0) chol_strip_update<B + 1, 8>(acc, Ubuf, warp, c0, lq, lr);
+        if constexpr (B < 7) {
+            if (bsrc != nullptr) chol_strip_lookahead<B + 1>(acc, ua, bsrc, warp < 4, c0, lq, lr);
+        }
     }
     strip_bar_sync(2);       // W is there; nobody reads the previous new rows any more
     // 2. new rows = W R
@@ -270,10 +299,11 @@ __device__ __forceinline__ void chol_strip_block(double (&acc)[8][2][2], double*
 template <int... Bs>
 __device__ __forceinline__ void chol_strip_blocks(double (&acc)[8][2][2], double* Rbuf, double* Ubuf, double* Wbuf,
                                                   int warp, int lane, int k0, bool reporter, int32_t* status,
+                                                  const double* ua, const double* bsrc,
                                                   std::integer_sequence<int, Bs...>) {
     chol_strip_publish<0>(acc, Rbuf, 16 * warp, lane >> 2, lane & 3);
     if (warp == 0) strip_bar_sync(1); else strip_bar_arrive(1);
-    (chol_strip_block<Bs>(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, reporter, status), ...);
+    (chol_strip_block<Bs>(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, reporter, status, ua, bsrc), ...);
 }
 
 // Factorises the diagonal block of A at k0 and applies the same row operations to 64 panel columns with it: columns
@@ -289,7 +319,11 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
                                            int pc0, bool identity, bool write_diag, double* __restrict__ D,
                                            double* smem, int vec16, int32_t* status, const double* upd_a,
                                            const double* upd_b) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // "warp" below is the index of the 16-column group a warp owns, not its hardware number.  Warps w and w + 4 share a
+    // scheduler; warp 0 (group 0, the chain) is paired with the next lightest group (diagonal columns 16 .. 31, whose
+    // fragments below row 32 are unused) and the heavier groups are spread over the other schedulers:
+    // hardware warp 0 1 2 3 4 5 6 7 -> group 0 2 3 6 1 4 5 7.
+    const int lane = threadIdx.x & 31, warp = (int)((0x75416320u >> (4 * (threadIdx.x >> 5))) & 7u);
     const int lq = lane >> 2, lr = lane & 3;
     double* Rbuf = smem;
     double* Ubuf = smem + 8 * kStripLd;
@@ -332,42 +366,20 @@ __device__ __forceinline__ void chol_strip(double* __restrict__ A, int64_t ld, i
                 }
             }
     }
+    // Look-ahead update with the block row above: only the first fragment row (and warp 0's second: warp 0 runs the
+    // chains and has no other rows in use) is brought up to date here; the others follow inside the strip, each while
+    // warp 0 works on the mini-block before it.
+    const double* bsrc = nullptr;
     if (upd_a != nullptr) {
         cp_async_wait<0>();
         __syncthreads();
-        const double* bsrc = is_diag ? upd_a + 16 * warp : (upd_b != nullptr ? upd_b + 16 * (warp - 4) : nullptr);
+        bsrc = is_diag ? upd_a + 16 * warp : (upd_b != nullptr ? upd_b + 16 * (warp - 4) : nullptr);
         if (bsrc != nullptr) {
-            double prod[8][2][2];
-#pragma unroll
-            for (int rb = 0; rb < 8; ++rb)
-#pragma unroll
-                for (int cb = 0; cb < 2; ++cb) prod[rb][cb][0] = prod[rb][cb][1] = 0.0;
-#pragma unroll 2
-            for (int kk = 0; kk < kNB; kk += 4) {
-                double bf[2];
-#pragma unroll
-                for (int cb = 0; cb < 2; ++cb) bf[cb] = bsrc[(kk + lr) * kCholLd + 8 * cb + lq];
-#pragma unroll
-                for (int rb = 0; rb < 8; ++rb) {
-                    const double af = upd_a[(kk + lr) * kCholLd + 8 * rb + lq];
-#pragma unroll
-                    for (int cb = 0; cb < 2; ++cb) {
-                        // fragments of the diagonal block that lie entirely below the diagonal are never used
-                        if (is_diag && 8 * rb > sc0 + 8 * cb + 7) continue;
-                        dmma_884(prod[rb][cb][0], prod[rb][cb][1], af, bf[cb]);
-                    }
-                }
-            }
-#pragma unroll
-            for (int rb = 0; rb < 8; ++rb)
-#pragma unroll
-                for (int cb = 0; cb < 2; ++cb) {
-                    acc[rb][cb][0] -= prod[rb][cb][0];
-                    acc[rb][cb][1] -= prod[rb][cb][1];
-                }
+            chol_strip_lookahead<0>(acc, upd_a, bsrc, is_diag, sc0, lq, lr);
+            if (warp == 0) chol_strip_lookahead<1>(acc, upd_a, bsrc, is_diag, sc0, lq, lr);
         }
     }
-    chol_strip_blocks(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, write_diag && threadIdx.x == 0, status,
+    chol_strip_blocks(acc, Rbuf, Ubuf, Wbuf, warp, lane, k0, write_diag && threadIdx.x == 0, status, upd_a, bsrc,
                       std::make_integer_sequence<int, 8>());
     if (is_diag) {
         if (write_diag) {
@@ -617,14 +629,14 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         }
         const int next_items = strip_items(k + 1) > 0 ? strip_items(k + 1) : 1;
         // Look-ahead pays when giving up next_items CTAs lengthens the trailing phase by less than the strip phase and
-        // the extra grid barrier it saves: compare rounds of tiles (about 4 us each) with and without, plus about 19 us.
+        // the extra grid barrier it saves: compare rounds of tiles (about 4 us each) with and without, plus about 15 us.
         bool look_ahead = false;
         if (next_items < G) {
             const int m_la = nb - k - 2, m_nl = nb - k - 1;
             const int t_la = m_la * (m_la + 1) / 2 + (Wm != nullptr ? m_la * (k + 1) : 0);
             const int t_nl = m_nl * (m_nl + 1) / 2 + (Wm != nullptr ? m_nl * (k + 1) : 0);
             const int g_la = G - next_items;
-            look_ahead = 4 * ((t_la + g_la - 1) / g_la) <= 4 * ((t_nl + G - 1) / G) + 19;
+            look_ahead = 4 * ((t_la + g_la - 1) / g_la) <= 4 * ((t_nl + G - 1) / G) + 15;
         }
         if (look_ahead) {
             // Look-ahead: the first next_items CTAs bring their own strip of block row k + 1 up to date and factorise

@@ -569,7 +569,9 @@ inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p
     const int groups = cdiv(rows, kSweepRows);
     if (cudaMemsetAsync(flags, 0, ((size_t)groups + 1) * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     // every byte 0xFF is a NaN: "not published yet" for the owner of the next block, which polls the values themselves
-    if (cudaMemsetAsync(E, 0xFF, (size_t)rows * ld * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
+    if (cudaMemset2DAsync(E, (size_t)ld * sizeof(double), 0xFF, (size_t)n * sizeof(double), (size_t)rows, stream) !=
+        cudaSuccess)
+        return PTQ_ERR_CUDA;
     SweepParams prm;
     prm.Wp = Wp; prm.U = U; prm.E = E; prm.codes_p = codes_p; prm.scale = scale; prm.zero = zero;
     prm.rows = rows; prm.n = n; prm.bits = bits; prm.ld = ld;

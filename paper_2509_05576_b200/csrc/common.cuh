@@ -137,7 +137,7 @@ enum KernelId {
     K_DGEMM_LAUUM, K_EXTRACT_DIAG, K_MINMAX_GRID, K_SCORE_PARTIAL,
     K_SCORE_FINAL, K_RANK_SORT, K_PERM_CHECK, K_GATHER_SYM, K_GATHER_W, K_SWEEP_COOP, K_FINALIZE,
     K_DGEMM_LOSS, K_SUM_PARTIALS, K_SELFTEST, K_FP64_PROBE, K_DYN_AUX, K_DYN_GATHER,
-    K_DGEMM_DYN, K_PER_ROW, K_COUNT
+    K_DGEMM_DYN, K_PER_ROW, K_DGEMM_EQ11, K_COUNT
 };
 
 inline const char* kernel_name(int id) {
@@ -146,7 +146,7 @@ inline const char* kernel_name(int id) {
         "dgemm_lauum", "extract_diag",
         "minmax_grid", "score_partial", "score_final", "rank_sort", "perm_check", "gather_sym", "gather_w",
         "sweep_coop", "finalize", "dgemm_loss", "sum_partials", "selftest_wait", "fp64_probe", "dyn_aux", "dyn_gather",
-        "dgemm_dyn", "per_row"};
+        "dgemm_dyn", "per_row", "dgemm_eq11"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 
