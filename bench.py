@@ -232,7 +232,7 @@ def layer_set_totals(fp64_peak, flush, ws):
     from paper_2509_05576_b200 import layer_set_run as lsr
 
     def brief(res, per_layer=False):
-        out = {k: res[k] for k in ("n_layers", "weights", "total_ms", "weights_per_s", "stage_total_ms",
+        out = {k: res[k] for k in ("n_layers", "weights", "total_ms", "weights_per_s", "graph_total_ms", "stage_total_ms",
                                    "stage_roofline_frac")}
         if per_layer:
             out["layers"] = [{"layer": r["layer"], "ms": r["ms"], "stages_ms": r["stages_ms"],
@@ -240,10 +240,10 @@ def layer_set_totals(fp64_peak, flush, ws):
         return out
 
     sets = {}
-    sets["c3_resnet50_w4"] = brief(lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush))
+    sets["c3_resnet50_w4"] = brief(lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True))
     # the YOLOv5s-shaped layers at 8 and 4 bits share their inputs: run the two bit-widths of a layer back to back
     c4 = [s for pair in zip(wl.config4(bits=(8,)), wl.config4(bits=(4,))) for s in pair]
-    res4 = lsr.run_specs(c4, 2, fp64_peak=fp64_peak, ws=ws, flush=flush)
+    res4 = lsr.run_specs(c4, 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True)
     for b in (8, 4):
         rows = [r for r in res4["layers"] if r["bits"] == b]
         st = {}
@@ -253,7 +253,8 @@ def layer_set_totals(fp64_peak, flush, ws):
         ms = sum(r["ms"] for r in rows)
         wts = sum(r["rows"] * r["cols"] for r in rows)
         sets[f"c4_yolov5s_w{b}"] = {"n_layers": len(rows), "weights": wts, "total_ms": ms,
-                                    "weights_per_s": wts / (ms * 1e-3), "stage_total_ms": st}
+                                    "weights_per_s": wts / (ms * 1e-3),
+                                    "graph_total_ms": sum(r["graph_ms"] for r in rows), "stage_total_ms": st}
     sets["c4_yolov5s_w8"]["stage_roofline_frac_both_bit_widths"] = res4["stage_roofline_frac"]
     sets["c5_scaling_w3_w4_w8"] = brief(lsr.run_specs(wl.config5(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush),
                                         per_layer=True)

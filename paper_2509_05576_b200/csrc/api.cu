@@ -26,8 +26,8 @@ inline int grid_x_for(int n, int threads) {
 
 // The loss product is cut along k into as many slices as it takes to put about two CTAs on every SM.
 constexpr int kMaxGridY = 65535;
-constexpr int kSuperBlock = 512;          // columns swept per launch on tall, wide layers
-constexpr int kSuperBlockMinRows = 512;
+constexpr int kSuperBlock = 1024;         // columns swept per launch on tall, wide layers
+constexpr int kSuperBlockMinRows = 2048;
 constexpr int kLossMaxSplit = 8;
 int loss_ksplit(int rows, int cols) {
     const long ctas = (long)cdiv(rows, 64) * ((cdiv(cols, 64) + 1) / 2);
@@ -611,9 +611,9 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
 
     if (rows >= kSuperBlockMinRows && n >= 4 * kSuperBlock) {
         // Tall and wide layers: the deferred part of Eq. 11 dominates (rows cols^2 / 2 multiply-adds), and inside the sweep
-        // kernel it runs as 32 x 64 x 64 tiles.  The columns are therefore swept in super-blocks of 512; what a
+        // kernel it runs as 32 x 64 x 64 tiles.  The columns are therefore swept in super-blocks of 1024; what a
         // super-block owes to all later columns is applied by one large product, W[:, later] -= E[:, sb] U[sb, later],
-        // on 128 x 128 tiles with k = 512.
+        // on 128 x 128 tiles with k = 1024.
         for (int off = 0; off < n; off += kSuperBlock) {
             const int sb = n - off < kSuperBlock ? n - off : kSuperBlock;
             st = sweep_launch(Wp + off, U + (size_t)off * n + off, E + off, codes_p + off, scale, zero, rows, sb, bits,

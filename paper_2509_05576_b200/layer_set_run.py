@@ -49,11 +49,14 @@ def stage_work(spec):
     }
 
 
-def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP64_PEAK_TFLOPS, ws=None, flush=None):
+def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP64_PEAK_TFLOPS, ws=None, flush=None,
+              graphs=False):
     """Quantizes the given layers one after the other on the current stream and times every C-ABI call with CUDA
     events (L2 flushed before every timed repetition, median over the repetitions).  Consecutive specs that describe
     the same seeded layer at another bit-width reuse its inputs.  Returns the per-layer records, the set totals, the
-    per-stage totals and the per-stage roofline fractions of the whole set (sum of work / sum of time / peak)."""
+    per-stage totals and the per-stage roofline fractions of the whole set (sum of work / sum of time / peak).
+    graphs=True also captures every layer's path as a CUDA graph and times its replay (``graph_ms`` per layer,
+    ``graph_total_ms`` for the set): what a caller gets who does not issue the launches one by one."""
     hbm, bf16, src = _peaks()
     int8_peak = bf16 * INT8_OVER_BF16
     s = torch.cuda.current_stream()
@@ -93,13 +96,29 @@ def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP
                 "inverse": work["inverse"] / (st["inverse"] * 1e-3) / 1e12 / fp64_peak,
                 "sweep": work["sweep"] / (st["sweep"] * 1e-3) / 1e12 / fp64_peak}
         loss = float(bufs.loss.item())
+        graph_ms = None
+        if graphs:
+            lg = ptq.LayerGraph(Wd, Xd, spec.bits, spec.damp, score_mode=score_mode, bufs=bufs, ws=ws)
+            ts = []
+            for rep in range(reps + 1):
+                flush.fill_(rep)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(s)
+                lg.replay()
+                b.record(s)
+                torch.cuda.synchronize()
+                if rep:
+                    ts.append(a.elapsed_time(b))
+            ptq.check_status(bufs.status, spec.name + " (graph)")
+            graph_ms = float(np.median(ts))
+            del lg
         if not quiet:
             print(f"{spec.name:28s} {spec.rows:5d} {spec.cols:6d} {spec.n:5d} {spec.bits:2d} {total:9.3f} "
                   f"{spec.weights / total / 1e3:8.1f} {st['hessian']:7.3f} {st['inverse']:7.3f} "
                   f"{st['grid'] + st['order']:6.3f} {st['sweep']:7.3f} {100 * frac['hessian']:6.2f} "
                   f"{100 * frac['inverse']:8.2f} {100 * frac['sweep']:8.2f} {loss:12.5g}")
         rows_out.append({"layer": spec.name, "rows": spec.rows, "cols": spec.cols, "n": spec.n, "bits": spec.bits,
-                         "ms": total, "stages_ms": st, "roofline_frac": frac, "loss": loss})
+                         "ms": total, "stages_ms": st, "roofline_frac": frac, "loss": loss, "graph_ms": graph_ms})
         totals["weights"] += spec.weights
         totals["ms"] += total
         totals["loss"] += loss
@@ -110,7 +129,9 @@ def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP
     stage_frac = {"hessian": work_tot["hessian"] / (stage_tot["hessian"] * 1e-3) / 1e12 / int8_peak,
                   "inverse": work_tot["inverse"] / (stage_tot["inverse"] * 1e-3) / 1e12 / fp64_peak,
                   "sweep": work_tot["sweep"] / (stage_tot["sweep"] * 1e-3) / 1e12 / fp64_peak}
+    graph_total = sum(r["graph_ms"] for r in rows_out) if graphs else None
     return {"layers": rows_out, "n_layers": len(rows_out), "weights": totals["weights"], "total_ms": totals["ms"],
+            "graph_total_ms": graph_total,
             "weights_per_s": totals["weights"] / (totals["ms"] * 1e-3), "loss_sum": totals["loss"],
             "stage_total_ms": stage_tot, "stage_roofline_frac": stage_frac,
             "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak, "fp64_tflops": fp64_peak, "source": src}}
@@ -129,6 +150,7 @@ def main(argv=None):
     ap.add_argument("--score-mode", default="qerr", choices=sorted(SCORE_MODES),
                     help="column ordering: qerr (Eq. 10, the method's), prune (Eq. 8), err, w, none (no sorting)")
     ap.add_argument("--ascending", action="store_true", help="sort the scores ascending (the 'asc' keys of Sec. 4.1)")
+    ap.add_argument("--graphs", action="store_true", help="also time every layer's path replayed as one CUDA graph")
     args = ap.parse_args(argv)
     if not torch.cuda.is_available():
         raise RuntimeError("layer_set_run needs a CUDA device")
@@ -145,7 +167,7 @@ def main(argv=None):
     s = torch.cuda.current_stream()
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
     mode = SCORE_MODES[args.score_mode] | (ptq.SCORE_ASCENDING if args.ascending else 0)
-    res = run_specs(specs, args.reps, mode, quiet=False, flush=flush)
+    res = run_specs(specs, args.reps, mode, quiet=False, flush=flush, graphs=args.graphs)
     totals = {"ms": res["total_ms"]}
     overlapped = None
     if args.streams > 1:
@@ -190,6 +212,7 @@ def main(argv=None):
                       "loss_sum": res["loss_sum"], "overlapped": overlapped,
                       "layers": res["n_layers"], "weights": res["weights"],
                       "total_ms": res["total_ms"], "weights_per_s": res["weights_per_s"],
+                      "graph_total_ms": res["graph_total_ms"],
                       "stage_total_ms": res["stage_total_ms"], "stage_roofline_frac": res["stage_roofline_frac"],
                       "peaks": res["peaks"]}))
     return 0

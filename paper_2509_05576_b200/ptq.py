@@ -369,6 +369,33 @@ def quantize_layer_full(W, X, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG, sco
     return bufs
 
 
+class LayerGraph:
+    """The whole path of one layer captured once as a CUDA graph and replayed: for layers so small that launching
+    their twenty-odd kernels one by one from the host takes longer than running them.
+
+    The graph is tied to the tensors it was captured with (W, X, the LayerBuffers and the workspace): refill W and X
+    in place and call ``replay()``.  Warm up the same call once before capturing (the first call on a device sets
+    kernel attributes, which is not a stream operation)."""
+
+    def __init__(self, W, X, bits, damp=0.01, damp_mode=DAMP_REL_MEAN_DIAG, score_mode=SCORE_QERR, bufs=None, ws=None):
+        rows, cols = W.shape
+        self.bufs = bufs or LayerBuffers(rows, cols, W.device)
+        self.ws = ws or Workspace(W.device)
+        self.stream = torch.cuda.Stream(device=W.device)
+        args = (W, X, bits, damp, damp_mode, score_mode)
+        self.stream.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(self.stream):
+            quantize_layer_full(*args, bufs=self.bufs, ws=self.ws, stream=self.stream)       # warm-up, sizes the workspace
+        self.stream.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph, stream=self.stream):
+            quantize_layer_full(*args, bufs=self.bufs, ws=self.ws, stream=self.stream)
+
+    def replay(self):
+        self.graph.replay()
+        return self.bufs
+
+
 class HostStaging:
     """Device landing buffers and the copy stream used by ``quantize_layer_from_host`` (allocated once per shape)."""
 

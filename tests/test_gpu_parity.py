@@ -368,3 +368,25 @@ def test_sharded_entry_on_one_rank_equals_the_single_gpu_path():
     assert float(res["loss"].item()) == float(g["loss"][0])
     out = {k: res[k].cpu().numpy() for k in ("perm", "scale", "zero", "codes", "What", "loss")}
     assert assert_layer_parity(out, ref) == 0
+
+
+def test_layer_path_replayed_as_a_cuda_graph_matches_the_eager_path():
+    """The whole path of a layer captured once and replayed: same bits as the call-by-call path, and new inputs written
+    into the captured tensors give the new layer's result (checked against the oracle)."""
+    W, X = _layer(96, 200, 512, 1500)
+    g = gpu_layer(W, X, 4)
+    Wd, Xd = _cuda(W), _cuda(X)
+    lg = ptq.LayerGraph(Wd, Xd, 4)
+    bufs = lg.replay()
+    torch.cuda.synchronize()
+    ptq.check_status(bufs.status, "graph replay")
+    for k in ("H", "Hinv", "S", "perm", "codes", "What", "loss"):
+        assert np.array_equal(getattr(bufs, k).cpu().numpy(), g[k]), k
+    W2, X2 = _layer(96, 200, 512, 1501)
+    Wd.copy_(_cuda(W2)); Xd.copy_(_cuda(X2))
+    bufs = lg.replay()
+    torch.cuda.synchronize()
+    ptq.check_status(bufs.status, "graph replay 2")
+    ref = oracle_layer(W2, X2, 4)
+    out = {k: getattr(bufs, k).cpu().numpy() for k in ("perm", "scale", "zero", "codes", "What", "loss")}
+    assert assert_layer_parity(out, ref) == 0
