@@ -201,30 +201,6 @@ def algorithmic_work(spec):
     }
 
 
-def measure_fp64_peak(ptq, torch, stream):
-    """Float64 throughput of this GPU, measured in this run with the library's probe kernels (eight independent
-    chains of FMAs, or of tensor-core m8n8k4 MMAs, per thread and nothing else): best of five launches of each kind,
-    timed with CUDA events on the launching stream after two warm-up launches."""
-    sink = torch.zeros(1, dtype=torch.float64, device="cuda")
-    out = {}
-    for kind, name, iters in ((0, "dfma", 100000), (1, "dmma", 20000)):
-        best = 0.0
-        for rep in range(7):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            flops = ptq.fp64_probe(kind, iters, sink, stream)
-            b.record(stream)
-            torch.cuda.synchronize()
-            if rep >= 2:
-                best = max(best, flops / (a.elapsed_time(b) * 1e-3) / 1e12)
-        out[name + "_tflops"] = best
-    out["fp64_tflops"] = max(out["dfma_tflops"], out["dmma_tflops"])
-    out["bound_tflops"] = FP64_PEAK_BOUND_TFLOPS
-    out["how"] = ("ptq_fp64_probe: 4 CTAs x 256 threads per SM, 8 independent chains per thread, 100000 (FMA) / 20000 (MMA) "
-                  "rounds, best of 5 launches, CUDA events; bound = 148 SMs x 64 FMA/clk x 2 x 1.965 GHz")
-    return out
-
-
 def layer_set_totals(fp64_peak, flush, ws):
     """The configurations beyond the single bench layer, measured in this run: the ResNet-50-shaped set (4-bit), the
     YOLOv5s-shaped set (8- and 4-bit) and the scaling shapes at 3, 4 and 8 bits.  Per set: total ms, weights/s, per-stage
@@ -240,7 +216,8 @@ def layer_set_totals(fp64_peak, flush, ws):
         return out
 
     sets = {}
-    sets["c3_resnet50_w4"] = brief(lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True))
+    sets["c3_resnet50_w4"] = brief(lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True),
+                                   per_layer=True)
     # the YOLOv5s-shaped layers at 8 and 4 bits share their inputs: run the two bit-widths of a layer back to back
     c4 = [s for pair in zip(wl.config4(bits=(8,)), wl.config4(bits=(4,))) for s in pair]
     res4 = lsr.run_specs(c4, 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True)
@@ -363,7 +340,8 @@ def run_ours(args):
     kernels = {k: {"ms_per_step": ms / prof_steps, "launches_per_step": cnt // prof_steps} for k, (ms, cnt) in prof.items()}
     dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     peaks = load_peaks()
-    peaks["fp64"] = measure_fp64_peak(ptq, torch, stream)
+    from paper_2509_05576_b200.layer_set_run import measure_fp64_peak
+    peaks["fp64"] = measure_fp64_peak(stream)
     peaks["fp64_tflops"] = peaks["fp64"]["fp64_tflops"]
     work = algorithmic_work(spec)
     per_kernel = kernel_rooflines(kernels, work, peaks)
@@ -439,6 +417,24 @@ def run_ours(args):
     if world == 1 and not args.no_sets:
         del Wd, Xd
         layer_sets = layer_set_totals(peaks["fp64_tflops"], flush, ws)
+        if not args.no_cpu_baseline:
+            # the oracle on a bounded sample of the ResNet-50-shaped set: every layer of at most 2304 columns (51 of the
+            # 54; the three 512 x 4608 layers alone would take the oracle longer than all the others together)
+            sample = [sp for sp in wl.config3() if sp.cols <= 2304]
+            cpu_s = 0.0
+            for sp in sample:
+                Ws, Xs = wl.make_layer(sp)
+                t0 = time.perf_counter()
+                oracle.run_layer(Ws, Xs, sp.bits, sp.damp)
+                cpu_s += time.perf_counter() - t0
+            names = {sp.name for sp in sample}
+            c3 = layer_sets["c3_resnet50_w4"]
+            gpu_ms = sum(r["ms"] for r in c3["layers"] if r["layer"] in names)
+            wts = sum(sp.weights for sp in sample)
+            c3["cpu_baseline"] = {"value": wts / cpu_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                                  "sample": f"the {len(sample)} layers of the set with at most 2304 columns "
+                                            f"({wts} weights), one pass each, {cpu_s:.1f} s",
+                                  "gpu_ms_on_the_same_sample": gpu_ms}
 
     if rank == 0:
         print(json.dumps({

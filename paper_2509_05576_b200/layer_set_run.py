@@ -24,7 +24,7 @@ import torch
 from . import ptq
 from . import workloads as wl
 
-FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12
+FP64_PEAK_TFLOPS = 148 * 64 * 2 * 1.965e9 / 1e12      # stated upper bound: 148 SMs x 64 FP64 FMA / clk x 2 x 1.965 GHz
 SCORE_MODES = {"qerr": ptq.SCORE_QERR, "prune": ptq.SCORE_PRUNE, "err": ptq.SCORE_ERR, "w": ptq.SCORE_W,
                "none": ptq.SCORE_NONE}
 INT8_OVER_BF16 = 2.0
@@ -37,6 +37,31 @@ def _peaks():
             p = json.load(f)
         return p["hbm_gbs"], p["bf16_tflops"], "measured"
     return 6650.0, 1590.0, "fallback"
+
+
+def measure_fp64_peak(stream=None):
+    """Float64 throughput of this GPU, measured with the library's probe kernels (eight independent chains of FMAs, or
+    of tensor-core m8n8k4 MMAs, per thread and nothing else): best of five launches of each kind, timed with CUDA
+    events on the launching stream after two warm-up launches."""
+    stream = stream or torch.cuda.current_stream()
+    sink = torch.zeros(1, dtype=torch.float64, device="cuda")
+    out = {}
+    for kind, name, iters in ((0, "dfma", 100000), (1, "dmma", 20000)):
+        best = 0.0
+        for rep in range(7):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            flops = ptq.fp64_probe(kind, iters, sink, stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            if rep >= 2:
+                best = max(best, flops / (a.elapsed_time(b) * 1e-3) / 1e12)
+        out[name + "_tflops"] = best
+    out["fp64_tflops"] = max(out["dfma_tflops"], out["dmma_tflops"])
+    out["bound_tflops"] = FP64_PEAK_TFLOPS
+    out["how"] = ("ptq_fp64_probe: 4 CTAs x 256 threads per SM, 8 independent chains per thread, 100000 (FMA) / 20000 (MMA) "
+                  "rounds, best of 5 launches, CUDA events; bound = 148 SMs x 64 FMA/clk x 2 x 1.965 GHz")
+    return out
 
 
 def stage_work(spec):
@@ -167,7 +192,9 @@ def main(argv=None):
     s = torch.cuda.current_stream()
     flush = torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
     mode = SCORE_MODES[args.score_mode] | (ptq.SCORE_ASCENDING if args.ascending else 0)
-    res = run_specs(specs, args.reps, mode, quiet=False, flush=flush, graphs=args.graphs)
+    fp64 = measure_fp64_peak(s)
+    res = run_specs(specs, args.reps, mode, quiet=False, flush=flush, graphs=args.graphs, fp64_peak=fp64["fp64_tflops"])
+    res["peaks"]["fp64_measured"] = fp64
     totals = {"ms": res["total_ms"]}
     overlapped = None
     if args.streams > 1:
