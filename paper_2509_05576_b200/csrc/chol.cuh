@@ -149,6 +149,7 @@ __device__ __forceinline__ void chol_load_block(double* dst, const double* __res
 // to warp 0 (the others only arrive), named barrier 2 hands W to everybody.
 // ------------------------------------------------------------------------------------------------------------
 constexpr int kStripLd = 132;                                            // row stride of the 8-row panels
+constexpr int kStripCostTiles = 4;                                       // a strip takes about as long as four trailing tiles
 constexpr int kStripSmemDoubles = 2 * 8 * kStripLd + 64;
 static_assert(kStripSmemDoubles <= 2 * 2 * kNB * kCholLd, "the strip panels alias the trailing-phase operand buffers");
 
@@ -532,21 +533,42 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
             __syncthreads();     // the panel buffers are reused by the next repetition and by the trailing phase
         }
     };
-    // Trailing tiles of block row k restricted to target rows >= row_base, processed by the CTAs cta_first .. G - 1.
+    // Trailing tiles of block row k restricted to target rows >= row_base.
     //   tiles of A: (i, j), row_base <= i <= j: A[i][j] -= U[k][i]^T U[k][j]
     //   tiles of W: (i, c), row_base <= i, c <= k:  W[i][c] -= U[k][i]^T W[k][c]       (row-major lists, A first)
-    auto trailing_phase = [&](int k, int row_base, int cta_first) {
+    // The CTAs 0 .. n_strip - 1 come here after a strip of the next block row (look-ahead), which costs them about as
+    // much as kStripCostTiles tiles: they take correspondingly fewer pieces, from the end of the list, so that all CTAs
+    // finish at about the same time.
+    auto trailing_phase = [&](int k, int row_base, int n_strip) {
         const int k0 = k * kNB;
         const int m = nb - row_base;
         const int TA = m * (m + 1) / 2;
         const int TW = Wm != nullptr ? m * (k + 1) : 0;
         const int T = TA + TW;
-        const int Gt = G - cta_first, me = (int)blockIdx.x - cta_first;
-        if (me < 0 || T <= 0) return;
+        if (T <= 0) return;
         // tiles are cut into 64 / H row pieces so that a short tile list still spreads over the grid
-        const int lgH = 4 * T <= Gt ? 4 : (2 * T <= Gt ? 5 : 6);
+        const int lgH = 4 * T <= G ? 4 : (2 * T <= G ? 5 : 6);
         const int lgP = 6 - lgH;
         const int TP = T << lgP;
+        const int S = n_strip < G ? n_strip : G, N = G - S;
+        int ps = 0;
+        if (S > 0) {
+            const int cs = kStripCostTiles << lgP;
+            const int target = (TP + S * cs + G - 1) / G;
+            ps = target > cs ? target - cs : 0;
+            if (N == 0) ps = (TP + S - 1) / S;
+        }
+        const int TPn = TP - S * ps > 0 ? TP - S * ps : 0;
+        const int pn = N > 0 ? (TPn + N - 1) / N : 0;
+        int tp_beg, tp_end;
+        if ((int)blockIdx.x >= S) {
+            tp_beg = ((int)blockIdx.x - S) * pn;
+            tp_end = tp_beg + pn < TPn ? tp_beg + pn : TPn;
+        } else {
+            tp_beg = TPn + (int)blockIdx.x * ps;
+            tp_end = tp_beg + ps < TP ? tp_beg + ps : TP;
+        }
+        if (tp_beg >= tp_end) return;
         struct Piece { double* C; const double* Bsrc; int i0, j0, tri; };
         // pieces are asked for in ascending order, so the row of the triangular list is found by walking on from the
         // row of the previous piece
@@ -574,8 +596,6 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         // operand then stays where it is and only B is fetched.
         double* abuf = opnd;                                  // [2][64][kCholLd]
         double* bbuf = opnd + 2 * kNB * kCholLd;              // [2][64][kCholLd]
-        const int per = (TP + Gt - 1) / Gt;
-        const int tp_beg = me * per, tp_end = tp_beg + per < TP ? tp_beg + per : TP;
         int stage = 0, a_slot = 0, a_next = 0;
         Piece cur{}, nxt{};
         if (tp_beg < tp_end) {
@@ -628,16 +648,10 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
             continue;
         }
         const int next_items = strip_items(k + 1) > 0 ? strip_items(k + 1) : 1;
-        // Look-ahead pays when giving up next_items CTAs lengthens the trailing phase by less than the strip phase and
-        // the extra grid barrier it saves: compare rounds of tiles (about 4 us each) with and without, plus about 15 us.
-        bool look_ahead = false;
-        if (next_items < G) {
-            const int m_la = nb - k - 2, m_nl = nb - k - 1;
-            const int t_la = m_la * (m_la + 1) / 2 + (Wm != nullptr ? m_la * (k + 1) : 0);
-            const int t_nl = m_nl * (m_nl + 1) / 2 + (Wm != nullptr ? m_nl * (k + 1) : 0);
-            const int g_la = G - next_items;
-            look_ahead = 4 * ((t_la + g_la - 1) / g_la) <= 4 * ((t_nl + G - 1) / G) + 15;
-        }
+        // Look-ahead whenever every strip item of the next block row finds a CTA of its own: those CTAs factorise their
+        // strip at once and then join the trailing tiles with a reduced share, so nobody idles and one grid barrier per
+        // block row is saved.
+        const bool look_ahead = next_items <= G;
         if (look_ahead) {
             // Look-ahead: the first next_items CTAs bring their own strip of block row k + 1 up to date and factorise
             // it at once, while the other CTAs apply block row k to the rows below k + 1.
@@ -655,9 +669,8 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
                 chol_strip(A, ld, n, (k + 1) * kNB, P, pc0, ident, g == 0, Dbuf + (size_t)(k + 1) * kNB * kNB, opnd, vec16,
                            status, ua, need_b ? ub : nullptr);
                 __syncthreads();
-            } else {
-                trailing_phase(k, k + 2, next_items);
             }
+            trailing_phase(k, k + 2, next_items);
         } else {
             trailing_phase(k, k + 1, 0);
             ++epoch;
