@@ -536,10 +536,10 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
     // Trailing tiles of block row k restricted to target rows >= row_base.
     //   tiles of A: (i, j), row_base <= i <= j: A[i][j] -= U[k][i]^T U[k][j]
     //   tiles of W: (i, c), row_base <= i, c <= k:  W[i][c] -= U[k][i]^T W[k][c]       (row-major lists, A first)
-    // The CTAs 0 .. n_strip - 1 come here after a strip of the next block row (look-ahead), which costs them about as
-    // much as kStripCostTiles tiles: they take correspondingly fewer pieces, from the end of the list, so that all CTAs
-    // finish at about the same time.
-    auto trailing_phase = [&](int k, int row_base, int n_strip) {
+    // In look-ahead mode the CTAs come here after `strips_b` strips of the next block row, the CTAs 0 .. n_more - 1 after
+    // one more; a strip costs about as much as kStripCostTiles tiles, so they take correspondingly fewer pieces (the
+    // busier CTAs from the end of the list) and all CTAs finish at about the same time.
+    auto trailing_phase = [&](int k, int row_base, int n_more, int strips_b) {
         const int k0 = k * kNB;
         const int m = nb - row_base;
         const int TA = m * (m + 1) / 2;
@@ -550,12 +550,14 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         const int lgH = 4 * T <= G ? 4 : (2 * T <= G ? 5 : 6);
         const int lgP = 6 - lgH;
         const int TP = T << lgP;
-        const int S = n_strip < G ? n_strip : G, N = G - S;
+        const int S = n_more < G ? n_more : G, N = G - S;
+        const int cs = kStripCostTiles << lgP;
+        const int cost_a = (strips_b + 1) * cs, cost_b = strips_b * cs;
         int ps = 0;
         if (S > 0) {
-            const int cs = kStripCostTiles << lgP;
-            const int target = (TP + S * cs + G - 1) / G;
-            ps = target > cs ? target - cs : 0;
+            const long work = (long)TP + (long)S * cost_a + (long)N * cost_b;
+            const int target = (int)((work + G - 1) / G);
+            ps = target > cost_a ? target - cost_a : 0;
             if (N == 0) ps = (TP + S - 1) / S;
         }
         const int TPn = TP - S * ps > 0 ? TP - S * ps : 0;
@@ -644,39 +646,28 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         if (!grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) break;
         // Block row k is final; the updates of block rows < k have been applied everywhere.
         if (k + 1 >= nbs) {                  // last factorised block row of a partial run: its update only
-            trailing_phase(k, k + 1, 0);
+            trailing_phase(k, k + 1, 0, 0);
             continue;
         }
         const int next_items = strip_items(k + 1) > 0 ? strip_items(k + 1) : 1;
-        // Look-ahead whenever every strip item of the next block row finds a CTA of its own: those CTAs factorise their
-        // strip at once and then join the trailing tiles with a reduced share, so nobody idles and one grid barrier per
-        // block row is saved.
-        const bool look_ahead = next_items <= G;
-        if (look_ahead) {
-            // Look-ahead: the first next_items CTAs bring their own strip of block row k + 1 up to date and factorise
-            // it at once, while the other CTAs apply block row k to the rows below k + 1.
-            if ((int)blockIdx.x < next_items) {
-                const int g = blockIdx.x;
-                double* P; int pc0; bool ident;
-                strip_item(k + 1, g, P, pc0, ident);
-                double* ua = opnd + 2 * kNB * kCholLd;        // beyond the strip's own panel buffers
-                double* ub = ua + kNB * kCholLd;
-                const bool need_b = P != nullptr && !ident;
-                __syncthreads();
-                chol_load_block(ua, A, ld, n, k * kNB, (k + 1) * kNB, 6, vec16);
-                if (need_b) chol_load_block(ub, P, ld, n, k * kNB, pc0, 6, vec16);
-                cp_async_commit();
-                chol_strip(A, ld, n, (k + 1) * kNB, P, pc0, ident, g == 0, Dbuf + (size_t)(k + 1) * kNB * kNB, opnd, vec16,
-                           status, ua, need_b ? ub : nullptr);
-                __syncthreads();
-            }
-            trailing_phase(k, k + 2, next_items);
-        } else {
-            trailing_phase(k, k + 1, 0);
-            ++epoch;
-            if (!grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) break;
-            strip_phase(k + 1);
+        // Look-ahead: the CTAs factorise the strips of block row k + 1 first (item g by CTA g mod G; each brings its
+        // strip up to date with block row k itself) and then join the trailing tiles of block row k below row k + 1 with
+        // a share reduced by what their strips cost, so nobody idles and there is one grid barrier per block row.
+        for (int g = blockIdx.x; g < next_items; g += G) {
+            double* P; int pc0; bool ident;
+            strip_item(k + 1, g, P, pc0, ident);
+            double* ua = opnd + 2 * kNB * kCholLd;        // beyond the strip's own panel buffers
+            double* ub = ua + kNB * kCholLd;
+            const bool need_b = P != nullptr && !ident;
+            __syncthreads();
+            chol_load_block(ua, A, ld, n, k * kNB, (k + 1) * kNB, 6, vec16);
+            if (need_b) chol_load_block(ub, P, ld, n, k * kNB, pc0, 6, vec16);
+            cp_async_commit();
+            chol_strip(A, ld, n, (k + 1) * kNB, P, pc0, ident, g == 0, Dbuf + (size_t)(k + 1) * kNB * kNB, opnd, vec16,
+                       status, ua, need_b ? ub : nullptr);
+            __syncthreads();
         }
+        trailing_phase(k, k + 2, next_items % G, next_items / G);
     }
     cp_async_wait<0>();
     // the diagonal factors move from the side buffer into A once nobody reads the original diagonal blocks any more
