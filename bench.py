@@ -233,6 +233,11 @@ def layer_set_totals(fp64_peak, flush, ws):
                                     "weights_per_s": wts / (ms * 1e-3),
                                     "graph_total_ms": sum(r["graph_ms"] for r in rows), "stage_total_ms": st}
     sets["c4_yolov5s_w8"]["stage_roofline_frac_both_bit_widths"] = res4["stage_roofline_frac"]
+    # independent layers of a set overlapped on four streams (the small layers leave most SMs idle on their own)
+    sets["c3_resnet50_w4"]["overlapped_4_streams_ms"] = lsr.run_overlapped(wl.config3(), 4, 2, flush=flush)["set_ms"]
+    for b in (8, 4):
+        sets[f"c4_yolov5s_w{b}"]["overlapped_4_streams_ms"] = lsr.run_overlapped(wl.config4(bits=(b,)), 4, 2,
+                                                                                 flush=flush)["set_ms"]
     sets["c5_scaling_w3_w4_w8"] = brief(lsr.run_specs(wl.config5(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush),
                                         per_layer=True)
     return sets

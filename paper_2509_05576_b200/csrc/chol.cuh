@@ -708,7 +708,12 @@ inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* 
         return (e == cudaSuccess && per_sm < 1) ? cudaErrorLaunchOutOfResources : e;
     });
     if (st) return st;
-    const int grid = dev->sms;   // one CTA per SM: the cooperative launch guarantees that all of them are resident
+    // One CTA per SM (the cooperative launch guarantees that all of them are resident); a matrix of a few block rows
+    // gets only as many CTAs as it ever has work items, which makes its grid barriers cheaper and leaves SMs to kernels
+    // of other streams.
+    const int nbr = (n + kNB - 1) / kNB;
+    const long items = (long)nbr * (nbr + 1) / 2 + (Wm != nullptr ? (long)nbr * nbr : 0);
+    const int grid = items < dev->sms ? (int)(items < 1 ? 1 : items) : dev->sms;
     if (cudaMemsetAsync(bar, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int64_t ld = n;
     int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;

@@ -565,7 +565,13 @@ inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p
         return (e == cudaSuccess && per_sm < 1) ? cudaErrorLaunchOutOfResources : e;
     });
     if (st) return st;
-    const int grid = dev->sms;
+    // one CTA per SM; with few row groups only the CTAs that get a share of the blocks are launched
+    const int groups_l = cdiv(rows, kSweepRows), nb_l = cdiv(n, kNB);
+    int grid = dev->sms;
+    if (groups_l < grid) {
+        const int per = grid / groups_l < nb_l ? grid / groups_l : nb_l;
+        grid = groups_l * per;
+    }
     const int groups = cdiv(rows, kSweepRows);
     if (cudaMemsetAsync(flags, 0, ((size_t)groups + 1) * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     // every byte 0xFF is a NaN: "not published yet" for the owner of the next block, which polls the values themselves

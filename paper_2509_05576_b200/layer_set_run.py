@@ -162,6 +162,47 @@ def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP
             "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak, "fp64_tflops": fp64_peak, "source": src}}
 
 
+def run_overlapped(specs, n_streams, reps=2, score_mode=ptq.SCORE_QERR, flush=None):
+    """The whole set with independent layers dealt round-robin onto `n_streams` streams: every stream has its own
+    workspace, every layer its own output buffers, the inputs of all layers are put on the device first, one event pair
+    around the whole set (median of `reps` timed passes after one warm-up pass)."""
+    s = torch.cuda.current_stream()
+    flush = flush if flush is not None else torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
+    data = []
+    for spec in specs:
+        W, X = wl.make_layer(spec)
+        data.append((spec, torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()))
+    outs = [ptq.LayerBuffers(spec.rows, spec.cols) for spec in specs]      # one set of outputs per layer, kept
+    streams = [torch.cuda.Stream() for _ in range(n_streams)]
+    wss = [ptq.Workspace() for _ in streams]
+
+    def run_set():
+        for i, (spec, Wd, Xd) in enumerate(data):
+            k = i % len(streams)
+            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=score_mode,
+                                    bufs=outs[i], ws=wss[k], stream=streams[k])
+
+    times = []
+    for rep in range(reps + 1):
+        torch.cuda.synchronize()
+        flush.fill_(rep)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        for st_ in streams:
+            st_.wait_stream(s)
+        run_set()
+        for st_ in streams:
+            s.wait_stream(st_)
+        e1.record(s)
+        torch.cuda.synchronize()
+        if rep > 0:
+            times.append(e0.elapsed_time(e1))
+    for o, spec in zip(outs, specs):
+        ptq.check_status(o.status, spec.name)
+    return {"streams": n_streams, "set_ms": float(np.median(times)),
+            "loss_sum": float(sum(o.loss.item() for o in outs))}
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7])
@@ -198,41 +239,7 @@ def main(argv=None):
     totals = {"ms": res["total_ms"]}
     overlapped = None
     if args.streams > 1:
-        # independent layers on several streams: every stream has its own workspace and output buffers; the inputs
-        # of all layers are put on the device first; one event pair around the whole set
-        data = []
-        for spec in specs:
-            W, X = wl.make_layer(spec)
-            data.append((spec, torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()))
-        outs = [ptq.LayerBuffers(spec.rows, spec.cols) for spec in specs]      # one set of outputs per layer, kept
-        streams = [torch.cuda.Stream() for _ in range(args.streams)]
-        wss = [ptq.Workspace() for _ in streams]
-
-        def run_set():
-            for i, (spec, Wd, Xd) in enumerate(data):
-                k = i % len(streams)
-                ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=mode,
-                                        bufs=outs[i], ws=wss[k], stream=streams[k])
-
-        times = []
-        for rep in range(args.reps + 1):
-            torch.cuda.synchronize()
-            flush.fill_(rep)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(s)
-            for st_ in streams:
-                st_.wait_stream(s)
-            run_set()
-            for st_ in streams:
-                s.wait_stream(st_)
-            e1.record(s)
-            torch.cuda.synchronize()
-            if rep > 0:
-                times.append(e0.elapsed_time(e1))
-        for o, spec in zip(outs, specs):
-            ptq.check_status(o.status, spec.name)
-        overlapped = {"streams": args.streams, "set_ms": float(np.median(times)),
-                      "loss_sum": float(sum(o.loss.item() for o in outs))}
+        overlapped = run_overlapped(specs, args.streams, args.reps, mode, flush)
         print(f"whole set on {args.streams} streams: {overlapped['set_ms']:.2f} ms "
               f"(sum of the per-layer times on one stream: {totals['ms']:.2f} ms)")
     print(json.dumps({"config": args.config, "score_mode": args.score_mode, "ascending": bool(args.ascending),
