@@ -221,6 +221,21 @@ int ptq_quantize_layer_per_row(const float *W, int rows, int cols, int64_t ldw, 
  */
 int ptq_sort_scores(const double *S, int cols, int ascending, int32_t *perm, void *stream);
 
+/*
+ * C += alpha * A B^T for float64 operands, formed on the tensor cores from error-free int8 slices of the operands (the
+ * way ptq_hessian_accumulate forms H), to float64 accuracy: the product behind the deferred part of Eq. 11,
+ * W[:, later] -= E[:, block] U[block, later], exposed for cross-checks and for callers who want it on its own.
+ *   C [m x n] float64, row stride ldc, in/out
+ *   A [m x k] float64, row stride lda
+ *   B: b_is_kn = 0: [n x k], row stride ldb;  b_is_kn = 1: the matrix is stored as [k x n] (so C += alpha A B), stride ldb
+ *   k <= 16384 (PTQ_ERR_UNSUPPORTED beyond).  Rows of A / of B with wildly different magnitudes are fine (each has its
+ *   own power-of-two scale); within a row, entries below 2^-54 of the row's largest magnitude are rounded away.
+ * Workspace: ptq_gemm_nt_sliced_workspace_bytes(m, n, k).
+ */
+size_t ptq_gemm_nt_sliced_workspace_bytes(int m, int n, int k);
+int ptq_gemm_nt_sliced(double *C, int64_t ldc, const double *A, int64_t lda, const double *B, int64_t ldb, int b_is_kn,
+                       int m, int n, int k, double alpha, void *ws, size_t ws_bytes, int32_t *status, void *stream);
+
 const char *ptq_status_string(int code);
 int ptq_version(void);
 

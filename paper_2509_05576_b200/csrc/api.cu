@@ -7,6 +7,7 @@
 #include "gram.cuh"
 #include "dynamic.cuh"
 #include "perrow.cuh"
+#include "i8gemm.cuh"
 
 using namespace ptq;
 
@@ -219,6 +220,8 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
             add(((size_t)cdiv(rows, kSweepRows) + 1) * sizeof(unsigned));   // per-row-group progress counters of the sweep
             add(chol_scratch_doubles(cols) * sizeof(double));
+            if (rows >= kSuperBlockMinRows && cols >= 4 * kSuperBlock)
+                add(i8gemm_workspace_bytes(rows, cols, kSuperBlock));   // slices of E[:, sb] and U[sb, later]
             break;
         case PTQ_CALL_QUANTIZE_LAYER_PER_ROW:
             if (rows < 1) return 0;
@@ -521,6 +524,22 @@ int ptq_quantize_layer_per_row(const float* W, int rows, int cols, int64_t ldw, 
     return launch_status();
 }
 
+size_t ptq_gemm_nt_sliced_workspace_bytes(int m, int n, int k) {
+    if (m < 1 || n < 1 || k < 1) return 0;
+    return i8gemm_workspace_bytes(m, n, k);
+}
+
+int ptq_gemm_nt_sliced(double* C, int64_t ldc, const double* A, int64_t lda, const double* B, int64_t ldb, int b_is_kn,
+                       int m, int n, int k, double alpha, void* ws, size_t ws_bytes, int32_t* status, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!C || !A || !B || m < 1 || n < 1 || k < 1 || ldc < n || lda < k || ldb < (b_is_kn ? n : k))
+        return PTQ_ERR_INVALID_ARG;
+    if (k > kXMaxK) return PTQ_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < i8gemm_workspace_bytes(m, n, k)) return PTQ_ERR_WORKSPACE;
+    if (!aligned16(ws)) return PTQ_ERR_ALIGNMENT;
+    return i8gemm_nt(C, ldc, A, lda, B, ldb, b_is_kn ? 1 : 0, m, n, k, alpha, ws, status, stream);
+}
+
 int ptq_sort_scores(const double* S, int cols, int ascending, int32_t* perm, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!S || !perm || cols < 1) return PTQ_ERR_INVALID_ARG;
@@ -598,6 +617,8 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     unsigned* bar = cv.take<unsigned>(2);
     unsigned* sweep_flags = cv.take<unsigned>((size_t)cdiv(rows, kSweepRows) + 1);
     double* Dbuf = cv.take<double>(chol_scratch_doubles(n));
+    void* xws = (rows >= kSuperBlockMinRows && n >= 4 * kSuperBlock)
+                    ? static_cast<void*>(cv.take<char>(i8gemm_workspace_bytes(rows, n, kSuperBlock))) : nullptr;
 
     // flags and invperm are adjacent pieces of the workspace: clear both
     if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
@@ -613,20 +634,16 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
         // Tall and wide layers: the deferred part of Eq. 11 dominates (rows cols^2 / 2 multiply-adds), and inside the sweep
         // kernel it runs as 32 x 64 x 64 tiles.  The columns are therefore swept in super-blocks of 1024; what a
         // super-block owes to all later columns is applied by one large product, W[:, later] -= E[:, sb] U[sb, later],
-        // on 128 x 128 tiles with k = 1024.
+        // with k = 1024.
         for (int off = 0; off < n; off += kSuperBlock) {
             const int sb = n - off < kSuperBlock ? n - off : kSuperBlock;
             st = sweep_launch(Wp + off, U + (size_t)off * n + off, E + off, codes_p + off, scale, zero, rows, sb, bits,
                               sweep_flags, status, stream, n);
             if (st) return st;
             if (off + sb < n) {
-                GemmParams g = gemm_defaults();
-                g.A = E + off; g.lda = n; g.a_trans = 0;
-                g.B = U + (size_t)off * n + off + sb; g.ldb = n; g.b_trans = 0;
-                g.C = Wp + off + sb; g.ldc = n;
-                g.M = rows; g.N = n - off - sb; g.K = sb;
-                g.alpha = -1.0; g.beta = 1.0;
-                st = launch_dgemm(K_DGEMM_EQ11, g, 1, stream);
+                // W[:, later] -= E[:, sb] U[sb, later] on the int8 tensor path (i8gemm.cuh), float64-accurate
+                st = i8gemm_nt(Wp + off + sb, n, E + off, n, U + (size_t)off * n + off + sb, n, 1, rows, n - off - sb, sb,
+                               -1.0, xws, status, stream);
                 if (st) return st;
             }
         }

@@ -92,7 +92,7 @@ constexpr long long kSpinLimitCycles = 4000000000LL;
 // (cudaFuncSetAttribute is per device).  One table, one mutex; looked up with the caller's device current.
 // ---------------------------------------------------------------------------------------------------------
 constexpr int kMaxDevices = 64;
-enum SmemAttrSlot { SA_CHOL = 0, SA_SWEEP, SA_GRAM, SA_DGEMM, SA_SMALL, SA_PROBE, SA_COUNT };
+enum SmemAttrSlot { SA_CHOL = 0, SA_SWEEP, SA_GRAM, SA_DGEMM, SA_SMALL, SA_XGEMM, SA_COUNT };
 struct DeviceState {
     int sms = 0;
     int coop = 0;
@@ -137,7 +137,7 @@ enum KernelId {
     K_DGEMM_LAUUM, K_EXTRACT_DIAG, K_MINMAX_GRID, K_SCORE_PARTIAL,
     K_SCORE_FINAL, K_RANK_SORT, K_PERM_CHECK, K_GATHER_SYM, K_GATHER_W, K_SWEEP_COOP, K_FINALIZE,
     K_DGEMM_LOSS, K_SUM_PARTIALS, K_SELFTEST, K_FP64_PROBE, K_DYN_AUX, K_DYN_GATHER,
-    K_DGEMM_DYN, K_PER_ROW, K_DGEMM_EQ11, K_COUNT
+    K_DGEMM_DYN, K_PER_ROW, K_DGEMM_EQ11, K_X_SLICE, K_X_GEMM, K_COUNT
 };
 
 inline const char* kernel_name(int id) {
@@ -146,7 +146,7 @@ inline const char* kernel_name(int id) {
         "dgemm_lauum", "extract_diag",
         "minmax_grid", "score_partial", "score_final", "rank_sort", "perm_check", "gather_sym", "gather_w",
         "sweep_coop", "finalize", "dgemm_loss", "sum_partials", "selftest_wait", "fp64_probe", "dyn_aux", "dyn_gather",
-        "dgemm_dyn", "per_row", "dgemm_eq11"};
+        "dgemm_dyn", "per_row", "dgemm_eq11", "x_slice", "i8gemm_tcgen05"};
     return (id >= 0 && id < K_COUNT) ? names[id] : "unknown";
 }
 

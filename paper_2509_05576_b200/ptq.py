@@ -27,7 +27,7 @@ CALL_QUANTIZE_LAYER_PER_ROW = 6
 
 EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_conv", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
            "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_sensitivity_order_static", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
-           "ptq_sort_scores", "ptq_quantize_layer_dynamic", "ptq_quantize_layer_per_row", "ptq_selftest_wait_timeout", "ptq_fp64_probe",
+           "ptq_sort_scores", "ptq_gemm_nt_sliced", "ptq_gemm_nt_sliced_workspace_bytes", "ptq_quantize_layer_dynamic", "ptq_quantize_layer_per_row", "ptq_selftest_wait_timeout", "ptq_fp64_probe",
            "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
 
 
@@ -67,6 +67,10 @@ def lib():
         L.ptq_quantize_layer.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, vp, c_int, vp, vp, vp, vp, vp,
                                          c_size_t, vp, vp]
         L.ptq_sort_scores.argtypes = [vp, c_int, c_int, vp, vp]
+        L.ptq_gemm_nt_sliced_workspace_bytes.argtypes = [c_int, c_int, c_int]
+        L.ptq_gemm_nt_sliced_workspace_bytes.restype = c_size_t
+        L.ptq_gemm_nt_sliced.argtypes = [vp, c_int64, vp, c_int64, vp, c_int64, c_int, c_int, c_int, c_int, c_double, vp,
+                                         c_size_t, vp, vp]
         L.ptq_quantize_layer_per_row.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, vp, vp, vp, vp, vp,
                                                  vp, c_size_t, vp, vp]
         L.ptq_quantize_layer_dynamic.argtypes = [vp, c_int, c_int, c_int64, vp, vp, vp, c_int, c_int, c_int, vp, vp,
@@ -248,6 +252,17 @@ def sort_scores(S, perm, ascending=False, stream=None):
     _dev(S, torch.float64, "S"); _dev(perm, torch.int32, "perm")
     _check(lib().ptq_sort_scores(_ptr(S), S.numel(), 1 if ascending else 0, _ptr(perm), _stream(stream)),
            "ptq_sort_scores")
+
+
+def gemm_nt_sliced(C, A, B, alpha, ws, status, b_is_kn=False, stream=None):
+    """C += alpha * A @ B.T (b_is_kn: C += alpha * A @ B) for float64 device tensors, on the int8 tensor path."""
+    _dev(C, torch.float64, "C"); _dev(A, torch.float64, "A"); _dev(B, torch.float64, "B")
+    m, k = A.shape
+    n = B.shape[1] if b_is_kn else B.shape[0]
+    buf = ws.get(int(lib().ptq_gemm_nt_sliced_workspace_bytes(m, n, k)))
+    _check(lib().ptq_gemm_nt_sliced(_ptr(C), _rowmajor(C, "C"), _ptr(A), _rowmajor(A, "A"), _ptr(B), _rowmajor(B, "B"),
+                                    1 if b_is_kn else 0, m, n, k, float(alpha), _ptr(buf), buf.numel(), _ptr(status),
+                                    _stream(stream)), "ptq_gemm_nt_sliced")
 
 
 def selftest_wait_timeout(which, limit_cycles, ws, status, stream=None):
