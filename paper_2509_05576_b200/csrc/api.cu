@@ -29,6 +29,7 @@ inline int grid_x_for(int n, int threads) {
 constexpr int kMaxGridY = 65535;
 constexpr int kSuperBlock = 1024;         // columns swept per launch on tall, wide layers
 constexpr int kSuperBlockMinRows = 2048;
+constexpr int kSlicedMinCols = 3072;      // from here on the large float64 products run on the int8 tensor path
 constexpr int kLossMaxSplit = 8;
 int loss_ksplit(int rows, int cols) {
     const long ctas = (long)cdiv(rows, 64) * ((cdiv(cols, 64) + 1) / 2);
@@ -323,7 +324,18 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int st = cholesky_upper(R, n, V, Dbuf, bar, status, stream);
     if (st) return st;
-    st = lauum_lower(V, Hinv, n, stream);
+    if (n >= kSlicedMinCols && n <= kXMaxK && x_operand_bytes(n, n) <= (size_t)n * n * sizeof(double)) {
+        // Hinv = W^T W on the int8 tensor path: the columns of the lower-triangular W are sliced once (into R, which is
+        // free now) and serve as both operands; only k >= max(i, j) contributes, upper tiles computed and mirrored
+        Carver rv(R);
+        const XOperand w = x_slice_operand(rv, V, n, 1, n, n, stream);
+        XGemmParams prm{};
+        prm.C = Hinv; prm.ldc = n; prm.alpha = 1.0; prm.status = status;
+        prm.out_mode = X_OUT_SYM; prm.k_mode = X_K_FROM_MAX;
+        st = x_product(w, w, prm, stream);
+    } else {
+        st = lauum_lower(V, Hinv, n, stream);
+    }
     if (st) return st;
     { Launch l(K_EXTRACT_DIAG, stream); extract_diag_kernel<<<cdiv(n, 256), 256, 0, stream>>>(Hinv, n, Hinv_diag); }
     return launch_status();
@@ -659,7 +671,28 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
         finalize_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(codes_p, invperm, W, rows, n, ldw, scale,
                                                                            zero, codes, What, dW);
     }
-    if (want_loss) {
+    if (want_loss && rows >= kSuperBlockMinRows && n >= kSlicedMinCols && n <= kXMaxK &&
+        x_operand_bytes(rows, n) <= (size_t)rows * n * sizeof(double) &&
+        x_operand_bytes(n, n) <= (size_t)n * n * sizeof(double) &&
+        2 * (size_t)x_num_tiles(rows, n) <= loss_partials_count(rows, cols)) {
+        // 1/2 sum_ij dW_ij (dW H)_ij on the int8 tensor path.  H is symmetric: per 64-column block j the column blocks
+        // k < j count twice (they stand in for the blocks k > j as well) and the block k = j once, so two products
+        // with reduction epilogues, k before the tile's own block (weight 2 * 1/2) and k in it (weight 1/2).
+        // The slices of dW go where E was, those of H where U was: both are free now.
+        Carver ev(E), uv(U);
+        const XOperand a = x_slice_operand(ev, dW, n, 0, rows, n, stream);
+        const XOperand b = x_slice_operand(uv, H_undamped, n, 0, n, n, stream);
+        const int tiles = x_num_tiles(rows, n);
+        XGemmParams prm{};
+        prm.status = status; prm.out_mode = X_OUT_REDUCE; prm.D = dW; prm.ldd = n;
+        prm.k_mode = X_K_BEFORE_J; prm.alpha = 1.0; prm.partials = partials;
+        st = x_product(a, b, prm, stream);
+        if (st) return st;
+        prm.k_mode = X_K_OWN_J; prm.alpha = 0.5; prm.partials = partials + tiles;
+        st = x_product(a, b, prm, stream);
+        if (st) return st;
+        { Launch l(K_SUM_PARTIALS, stream); sum_partials_kernel<<<1, 256, 0, stream>>>(partials, 2 * tiles, 1.0, loss_out); }
+    } else if (want_loss) {
         // sum_ic dW_ic (dW H)_ic; H is symmetric, so for the 64-column block of c only k up to the end of that block is
         // summed and the blocks before it are doubled
         GemmParams g = gemm_defaults();

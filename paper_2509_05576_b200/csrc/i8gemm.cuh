@@ -42,6 +42,7 @@ inline size_t i8gemm_workspace_bytes(int m, int n, int k) {
     return align_up(i8gemm_plane_bytes(m, k)) + align_up(i8gemm_plane_bytes(n, k)) +
            align_up((size_t)(cdiv(m, 128) * 128) * sizeof(int32_t)) + align_up((size_t)(cdiv(n, 128) * 128) * sizeof(int32_t));
 }
+// Output / K-range modes and the slicing of one operand at a time: see XGemmParams, x_slice_operand, x_product below.
 
 __device__ __forceinline__ void x_pack4(const long long (&v)[4], uint32_t (&packed)[kXSlices]) {
 #pragma unroll
@@ -162,15 +163,41 @@ __global__ void __launch_bounds__(256) x_slice_cols_kernel(const double* __restr
     }
 }
 
+// Output modes: what the epilogue does with P = A B^T.
+enum { X_OUT_ADD = 0,        // C += alpha P
+       X_OUT_SYM = 1,        // C = alpha P on the tiles that touch the upper triangle, and C[j][i] = C[i][j] (A = B)
+       X_OUT_REDUCE = 2 };   // partials[tile] = alpha * sum_ij P_ij D_ij ; C is not touched
+// K ranges per tile (operands known to be zero outside them, or terms accounted for elsewhere).
+enum { X_K_ALL = 0,
+       X_K_FROM_MAX = 1,     // k >= max(i0, j0): A[i][k] = 0 for k < i and B[j][k] = 0 for k < j (a triangular factor)
+       X_K_BEFORE_J = 2,     // k < j0: the column blocks before the tile's own
+       X_K_OWN_J = 3 };      // j0 <= k < j0 + 64: the tile's own column block
 struct XGemmParams {
-    double* C;              // [m x n], row stride ldc: C += alpha * A B^T
+    double* C;              // [m x n], row stride ldc
     int64_t ldc;
     int m, n, k_pad;
     double alpha;
     const int32_t* sh_a;    // per row of A
     const int32_t* sh_b;    // per row of B
     int32_t* status;
+    int out_mode, k_mode;
+    const double* D;        // X_OUT_REDUCE: [m x n], row stride ldd
+    int64_t ldd;
+    double* partials;       // X_OUT_REDUCE: one per tile (0 for tiles without work)
 };
+
+// K blocks [kb0, kb1) of tile (bi, bj); an empty range or a tile below the diagonal (X_OUT_SYM) has no work at all.
+__device__ __forceinline__ bool x_tile_range(const XGemmParams& prm, int bi, int bj, int nkb, int& kb0, int& kb1) {
+    const int i0 = bi * kXTM, j0 = bj * kXTN;
+    kb0 = 0;
+    kb1 = nkb;
+    if (prm.out_mode == X_OUT_SYM && i0 > j0 + kXTN - 1) return false;
+    if (prm.k_mode == X_K_FROM_MAX) kb0 = (i0 > j0 ? i0 : j0) / kXKB;
+    else if (prm.k_mode == X_K_BEFORE_J) kb1 = j0 / kXKB;
+    else if (prm.k_mode == X_K_OWN_J) { kb0 = j0 / kXKB; kb1 = kb0 + 1; }
+    if (kb1 > nkb) kb1 = nkb;
+    return kb0 < kb1;
+}
 
 __global__ void __launch_bounds__(kXThreads, 1)
 i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__ CUtensorMap tmapB, XGemmParams prm) {
@@ -223,7 +250,9 @@ i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
                 const int bi = tile / tiles_n, bj = tile - bi * tiles_n;
-                for (int kb = 0; kb < nkb && ok; ++kb) {
+                int kb0, kb1;
+                if (!x_tile_range(prm, bi, bj, nkb, kb0, kb1)) continue;
+                for (int kb = kb0; kb < kb1 && ok; ++kb) {
                     ok = mbar_wait_bounded(empty_bar(stage), phase ^ 1u, abort_flag);
                     if (!ok) break;
                     const uint32_t sbase = base + stage * kXStageBytes;
@@ -254,15 +283,18 @@ i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__
             uint32_t phase = 0, acc_phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+                const int bi = tile / tiles_n, bj = tile - bi * tiles_n;
+                int kb0, kb1;
+                if (!x_tile_range(prm, bi, bj, nkb, kb0, kb1)) continue;
                 ok = mbar_wait_bounded(acc_empty, acc_phase ^ 1u, abort_flag);   // epilogue has drained TMEM
                 if (!ok) break;
                 tc_fence_after();
-                for (int kb = 0; kb < nkb && ok; ++kb) {
+                for (int kb = kb0; kb < kb1 && ok; ++kb) {
                     ok = mbar_wait_bounded(full_bar(stage), phase, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t sb = kDescLo + ((base + stage * kXStageBytes) >> 4);
-                    const uint32_t first = kb > 0 ? 1u : 0u;      // the first product of a group overwrites
+                    const uint32_t first = kb > kb0 ? 1u : 0u;    // the first product of a group overwrites
 #pragma unroll
                     for (int g = 0; g < kXGroups; ++g) {
 #pragma unroll
@@ -294,6 +326,11 @@ i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__
         bool ok = true;
         for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
             const int bi = tile / tiles_n, bj = tile - bi * tiles_n;
+            int kb0, kb1;
+            if (!x_tile_range(prm, bi, bj, nkb, kb0, kb1)) {
+                if (prm.out_mode == X_OUT_REDUCE && threadIdx.x == 64) prm.partials[tile] = 0.0;
+                continue;
+            }
             ok = mbar_wait_bounded(acc_full, acc_phase, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -337,6 +374,43 @@ i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__
             const int sh_i = row < prm.m ? prm.sh_a[row] : 0;
             const double fi = prm.alpha * __longlong_as_double((long long)(1023 + 24 - sh_i) << 52);
             const int orow = lane >> 4, ocol = lane & 15;
+            if (prm.out_mode == X_OUT_REDUCE) {
+                // sum_ij P_ij D_ij over the tile, in a fixed order: along the row in this lane, then over the lanes of
+                // the warp by a shuffle tree, then over the four warps in ascending order
+                double s = 0.0;
+                if (row < prm.m) {
+                    const double* drow = prm.D + (int64_t)row * prm.ldd + bj * kXTN;
+#pragma unroll
+                    for (int c = 0; c < kXTN; ++c) {
+                        const int col = bj * kXTN + c;
+                        if (col < prm.n) {
+                            const double fj = __longlong_as_double((long long)(1023 + 24 - prm.sh_b[col]) << 52);
+                            s = fma((v[c] * fi) * fj, drow[c], s);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+                if (lane == 0) my[0] = s;
+                asm volatile("bar.sync 1, 128;" ::: "memory");           // the four epilogue warps
+                if (quarter == 0 && lane == 0)
+                    prm.partials[tile] = ((epi[0] + epi[32 * 17]) + epi[2 * 32 * 17]) + epi[3 * 32 * 17];
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                continue;
+            }
+            if (prm.out_mode == X_OUT_SYM) {
+                // mirrored entries C[col][row]: consecutive lanes are consecutive rows, i.e. contiguous there
+                if (row < prm.m) {
+#pragma unroll
+                    for (int c = 0; c < kXTN; ++c) {
+                        const int col = bj * kXTN + c;
+                        if (col < prm.n) {
+                            const double fj = __longlong_as_double((long long)(1023 + 24 - prm.sh_b[col]) << 52);
+                            prm.C[(int64_t)col * prm.ldc + row] = (v[c] * fi) * fj;
+                        }
+                    }
+                }
+            }
 #pragma unroll
             for (int ch = 0; ch < kXTN / 16; ++ch) {
                 const int col0 = bj * kXTN + ch * 16;
@@ -351,7 +425,8 @@ i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__
                         const int grow = bi * kXTM + quarter * 32 + rr + orow;
                         if (grow < prm.m) {
                             double* dst = prm.C + (int64_t)grow * prm.ldc + col;
-                            *dst = fma(my[(rr + orow) * 17 + ocol], fj, *dst);
+                            const double pv = my[(rr + orow) * 17 + ocol] * fj;
+                            *dst = prm.out_mode == X_OUT_ADD ? *dst + pv : pv;
                         }
                     }
                 }
@@ -385,12 +460,34 @@ inline int x_make_map(CUtensorMap* m, int8_t* Q, int rows_pad, int k_pad, int bo
     return r == CUDA_SUCCESS ? PTQ_OK : PTQ_ERR_CUDA;
 }
 
-// C[m x n] += alpha * A B^T with A [m x k] (rows contiguous in k, stride lda) and B given either as [n x k]
-// (b_is_kn = 0, stride ldb) or as [k x n] (b_is_kn = 1: B^T is what is stored, stride ldb).  k <= kXMaxK.
-inline int i8gemm_nt(double* C, int64_t ldc, const double* A, int64_t lda, const double* B, int64_t ldb, int b_is_kn,
-                     int m, int n, int k, double alpha, void* ws, int32_t* status, cudaStream_t stream) {
-    if (m <= 0 || n <= 0 || k <= 0) return PTQ_OK;
-    if (k > kXMaxK) return PTQ_ERR_UNSUPPORTED;
+// Slices of one operand in the workspace: planes [7][rows_pad][k_pad] and the per-row shifts.
+struct XOperand {
+    int8_t* Q;
+    int32_t* sh;
+    int rows, k;
+};
+inline size_t x_operand_bytes(int rows, int k) {
+    return align_up(i8gemm_plane_bytes(rows, k)) + align_up((size_t)(cdiv(rows, 128) * 128) * sizeof(int32_t));
+}
+// X is [rows x k] (transposed = 0, row stride ld) or [k x rows] (transposed = 1: the operand's rows are X's columns).
+inline XOperand x_slice_operand(Carver& cv, const double* X, int64_t ld, int transposed, int rows, int k,
+                                cudaStream_t stream) {
+    const int rows_pad = cdiv(rows, 128) * 128, k_pad = cdiv(k, 128) * 128;
+    XOperand op;
+    op.Q = cv.take<int8_t>(i8gemm_plane_bytes(rows, k));
+    op.sh = cv.take<int32_t>(rows_pad);
+    op.rows = rows; op.k = k;
+    Launch l(K_X_SLICE, stream);
+    if (transposed)
+        x_slice_cols_kernel<<<rows_pad / 32, 256, 0, stream>>>(X, k, rows, ld, rows_pad, k_pad, op.Q, op.sh);
+    else
+        x_slice_rows_kernel<<<rows_pad, 256, 0, stream>>>(X, rows, k, ld, rows_pad, k_pad, op.Q, op.sh);
+    return op;
+}
+
+// The product of two sliced operands (A: m rows, B: n rows, same k <= kXMaxK) in the given output / K-range modes.
+inline int x_product(const XOperand& a, const XOperand& b, XGemmParams prm, cudaStream_t stream) {
+    if (a.k != b.k || a.k > kXMaxK) return PTQ_ERR_UNSUPPORTED;
     DeviceState* dev = nullptr;
     int st = current_device_state(&dev);
     if (st) return st;
@@ -398,35 +495,37 @@ inline int i8gemm_nt(double* C, int64_t ldc, const double* A, int64_t lda, const
         return cudaFuncSetAttribute(i8gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kXSmemBytes);
     });
     if (st) return st;
-    const int m_pad = cdiv(m, 128) * 128, n_pad = cdiv(n, 128) * 128, k_pad = cdiv(k, 128) * 128;
-    Carver cv(ws);
-    int8_t* QA = cv.take<int8_t>(i8gemm_plane_bytes(m, k));
-    int8_t* QB = cv.take<int8_t>(i8gemm_plane_bytes(n, k));
-    int32_t* shA = cv.take<int32_t>(m_pad);
-    int32_t* shB = cv.take<int32_t>(n_pad);
-    {
-        Launch l(K_X_SLICE, stream);
-        x_slice_rows_kernel<<<m_pad, 256, 0, stream>>>(A, m, k, lda, m_pad, k_pad, QA, shA);
-        if (b_is_kn)
-            x_slice_cols_kernel<<<n_pad / 32, 256, 0, stream>>>(B, k, n, ldb, n_pad, k_pad, QB, shB);
-        else
-            x_slice_rows_kernel<<<n_pad, 256, 0, stream>>>(B, n, k, ldb, n_pad, k_pad, QB, shB);
-    }
+    const int k_pad = cdiv(a.k, 128) * 128;
     CUtensorMap mapA, mapB;
-    st = x_make_map(&mapA, QA, m_pad, k_pad, kXTM);
+    st = x_make_map(&mapA, a.Q, cdiv(a.rows, 128) * 128, k_pad, kXTM);
     if (st) return st;
-    st = x_make_map(&mapB, QB, n_pad, k_pad, kXTN);
+    st = x_make_map(&mapB, b.Q, cdiv(b.rows, 128) * 128, k_pad, kXTN);
     if (st) return st;
-    XGemmParams prm;
-    prm.C = C; prm.ldc = ldc; prm.m = m; prm.n = n; prm.k_pad = k_pad; prm.alpha = alpha;
-    prm.sh_a = shA; prm.sh_b = shB; prm.status = status;
-    const int tiles = cdiv(m, kXTM) * cdiv(n, kXTN);
+    prm.m = a.rows; prm.n = b.rows; prm.k_pad = k_pad;
+    prm.sh_a = a.sh; prm.sh_b = b.sh;
+    const int tiles = cdiv(prm.m, kXTM) * cdiv(prm.n, kXTN);
     const int grid = tiles < dev->sms ? tiles : dev->sms;
     {
         Launch l(K_X_GEMM, stream);
         i8gemm_kernel<<<grid, kXThreads, kXSmemBytes, stream>>>(mapA, mapB, prm);
     }
     return launch_status();
+}
+inline int x_num_tiles(int m, int n) { return cdiv(m, kXTM) * cdiv(n, kXTN); }
+
+// C[m x n] += alpha * A B^T with A [m x k] (rows contiguous in k, stride lda) and B given either as [n x k]
+// (b_is_kn = 0, stride ldb) or as [k x n] (b_is_kn = 1: B^T is what is stored, stride ldb).  k <= kXMaxK.
+inline int i8gemm_nt(double* C, int64_t ldc, const double* A, int64_t lda, const double* B, int64_t ldb, int b_is_kn,
+                     int m, int n, int k, double alpha, void* ws, int32_t* status, cudaStream_t stream) {
+    if (m <= 0 || n <= 0 || k <= 0) return PTQ_OK;
+    if (k > kXMaxK) return PTQ_ERR_UNSUPPORTED;
+    Carver cv(ws);
+    const XOperand a = x_slice_operand(cv, A, lda, 0, m, k, stream);
+    const XOperand b = x_slice_operand(cv, B, ldb, b_is_kn, n, k, stream);
+    XGemmParams prm{};
+    prm.C = C; prm.ldc = ldc; prm.alpha = alpha; prm.status = status;
+    prm.out_mode = X_OUT_ADD; prm.k_mode = X_K_ALL;
+    return x_product(a, b, prm, stream);
 }
 
 }  // namespace ptq
