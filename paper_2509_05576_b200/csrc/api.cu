@@ -8,6 +8,7 @@
 #include "dynamic.cuh"
 #include "perrow.cuh"
 #include "i8gemm.cuh"
+#include "cholpanel.cuh"
 
 using namespace ptq;
 
@@ -204,6 +205,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(c * c * sizeof(double));
             add(2 * sizeof(unsigned));                      // grid barrier of the factorisation kernel
             add(chol_scratch_doubles(cols) * sizeof(double));
+            add(chol_panel_workspace_bytes(cols));          // operand slices of the panel updates (large matrices)
             break;
         case PTQ_CALL_SENSITIVITY_ORDER:
             if (rows < 1) return 0;
@@ -223,6 +225,7 @@ size_t ptq_workspace_bytes(int call_id, int rows, int cols, int n) {
             add(chol_scratch_doubles(cols) * sizeof(double));
             if (rows >= kSuperBlockMinRows && cols >= 4 * kSuperBlock)
                 add(i8gemm_workspace_bytes(rows, cols, kSuperBlock));   // slices of E[:, sb] and U[sb, later]
+            add(chol_panel_workspace_bytes(cols));
             break;
         case PTQ_CALL_QUANTIZE_LAYER_PER_ROW:
             if (rows < 1) return 0;
@@ -318,11 +321,12 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     double* V = cv.take<double>((size_t)n * n);
     unsigned* bar = cv.take<unsigned>(2);
     double* Dbuf = cv.take<double>(chol_scratch_doubles(n));
+    void* pws = chol_panel_workspace_bytes(n) ? static_cast<void*>(cv.take<char>(chol_panel_workspace_bytes(n))) : nullptr;
     { Launch l(K_LAMBDA, stream); lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status); }
     { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out); }
     // W = U^-T comes out of the factorisation sweep itself (V must start as zero)
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
-    int st = cholesky_upper(R, n, V, Dbuf, bar, status, stream);
+    int st = cholesky_upper_auto(R, n, V, Dbuf, bar, pws, status, stream);
     if (st) return st;
     if (n >= kSlicedMinCols && n <= kXMaxK && x_operand_bytes(n, n) <= (size_t)n * n * sizeof(double)) {
         // Hinv = W^T W on the int8 tensor path: the columns of the lower-triangular W are sliced once (into R, which is
@@ -631,6 +635,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     double* Dbuf = cv.take<double>(chol_scratch_doubles(n));
     void* xws = (rows >= kSuperBlockMinRows && n >= 4 * kSuperBlock)
                     ? static_cast<void*>(cv.take<char>(i8gemm_workspace_bytes(rows, n, kSuperBlock))) : nullptr;
+    void* pws = chol_panel_workspace_bytes(n) ? static_cast<void*>(cv.take<char>(chol_panel_workspace_bytes(n))) : nullptr;
 
     // flags and invperm are adjacent pieces of the workspace: clear both
     if (cudaMemsetAsync(flags, 0, (size_t)((char*)invperm - (char*)flags) + (size_t)n * sizeof(int32_t), stream) !=
@@ -639,7 +644,7 @@ int ptq_quantize_layer(const float* W, int rows, int cols, int64_t ldw, const do
     { Launch l(K_PERM_CHECK, stream); perm_check_kernel<<<cdiv(n, 256), 256, 0, stream>>>(perm, n, flags, invperm, status); }
     { Launch l(K_GATHER_SYM, stream); gather_sym_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(Hinv, perm, n, U); }
     { Launch l(K_GATHER_W, stream); gather_w_kernel<<<dim3(grid_x_for(n, 256), rows), 256, 0, stream>>>(W, rows, n, ldw, perm, Wp); }
-    int st = cholesky_upper(U, n, nullptr, Dbuf, bar, status, stream);   // blocked Eq. 12
+    int st = cholesky_upper_auto(U, n, nullptr, Dbuf, bar, pws, status, stream);   // blocked Eq. 12
     if (st) return st;
 
     if (rows >= kSuperBlockMinRows && n >= 4 * kSuperBlock) {

@@ -503,7 +503,8 @@ __device__ __forceinline__ void chol_trailing_piece(double* __restrict__ C, int6
 
 __global__ void __launch_bounds__(kCholThreads, 1)
 chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __restrict__ Dbuf, int n, int64_t ld,
-                 int vec16, unsigned* bar, int32_t* status, long long spin_limit, int nb_stop) {
+                 int vec16, unsigned* bar, int32_t* status, long long spin_limit, int k_first, int nb_stop,
+                 int row_limit) {
     extern __shared__ __align__(16) unsigned char chol_smem_raw[];
     double* opnd = reinterpret_cast<double*>(chol_smem_raw);                // [2 stages][2 operands][64][kCholLd]
     int* s_flag = reinterpret_cast<int*>(opnd + 2 * 2 * kNB * kCholLd);     // the strip panels alias opnd
@@ -533,7 +534,7 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
             __syncthreads();     // the panel buffers are reused by the next repetition and by the trailing phase
         }
     };
-    // Trailing tiles of block row k restricted to target rows >= row_base.
+    // Trailing tiles of block row k restricted to the target block rows row_base <= i < row_limit.
     //   tiles of A: (i, j), row_base <= i <= j: A[i][j] -= U[k][i]^T U[k][j]
     //   tiles of W: (i, c), row_base <= i, c <= k:  W[i][c] -= U[k][i]^T W[k][c]       (row-major lists, A first)
     // In look-ahead mode the CTAs come here after `strips_b` strips of the next block row, the CTAs 0 .. n_more - 1 after
@@ -541,9 +542,11 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
     // busier CTAs from the end of the list) and all CTAs finish at about the same time.
     auto trailing_phase = [&](int k, int row_base, int n_more, int strips_b) {
         const int k0 = k * kNB;
-        const int m = nb - row_base;
-        const int TA = m * (m + 1) / 2;
-        const int TW = Wm != nullptr ? m * (k + 1) : 0;
+        const int m = nb - row_base;                                        // tiles in the first target row
+        const int R = (row_limit < nb ? row_limit : nb) - row_base;         // target block rows
+        if (R <= 0) return;
+        const int TA = R * m - R * (R - 1) / 2;
+        const int TW = Wm != nullptr ? R * (k + 1) : 0;
         const int T = TA + TW;
         if (T <= 0) return;
         // tiles are cut into 64 / H row pieces so that a short tile list still spreads over the grid
@@ -635,13 +638,17 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
         cp_async_wait<0>();
     };
 
-    // nb_stop < nb: a partial factorisation.  Only the first nb_stop block rows are factorised; their updates are applied
-    // to everything below, so that the upper triangle of A[64 nb_stop :, 64 nb_stop :] ends up holding the Schur
-    // complement of the leading block (what Eq. 12 leaves after that many columns).
+    // The block rows k_first .. nb_stop - 1 are factorised (block row k_first must already carry the updates of all rows
+    // above it); their updates are applied to the target rows below row_limit.
+    //   k_first = 0, nb_stop = nb, row_limit = nb : the whole factorisation;
+    //   nb_stop < nb, row_limit = nb : a partial factorisation that leaves the Schur complement of the leading block in
+    //       the upper triangle of A[64 nb_stop :, 64 nb_stop :] (what Eq. 12 leaves after that many columns);
+    //   row_limit = nb_stop : a panel -- only its own block rows are touched; the caller applies the panel to the rows
+    //       below it in one product of depth 64 (nb_stop - k_first).
     const int nbs = nb_stop < nb ? nb_stop : nb;
-    const int steps = nbs < nb ? nbs : nb - 1;
-    strip_phase(0);
-    for (int k = 0; k < steps; ++k) {
+    const int steps = nbs < nb ? (row_limit > nbs ? nbs : nbs - 1) : nb - 1;
+    strip_phase(k_first);
+    for (int k = k_first; k < steps; ++k) {
         ++epoch;
         if (!grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) break;
         // Block row k is final; the updates of block rows < k have been applied everywhere.
@@ -673,7 +680,7 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
     // the diagonal factors move from the side buffer into A once nobody reads the original diagonal blocks any more
     ++epoch;
     if (grid_barrier(bar, epoch * (unsigned)G, s_flag, spin_limit)) {
-        for (int b = blockIdx.x; b < nbs; b += G)
+        for (int b = k_first + blockIdx.x; b < nbs; b += G)
             for (int idx = tid; idx < kNB * kNB; idx += kCholThreads) {
                 const int r = idx >> 6, c = idx & 63;
                 if (c >= r && b * kNB + c < n)
@@ -689,12 +696,15 @@ chol_coop_kernel(double* __restrict__ A, double* __restrict__ Wm, double* __rest
 // Sec. 5 item 1 asks for.
 // `bar` is 2 x uint32 of device scratch, Dbuf holds chol_scratch_doubles(n) doubles (the diagonal factors on their way).
 inline size_t chol_scratch_doubles(int n) { return (size_t)((n + kNB - 1) / kNB) * kNB * kNB; }
-// nb_stop > 0: factorise the first nb_stop block rows of 64 only and leave the Schur complement of that leading block in
-// the upper triangle of the rest (Wm must be null then).
+// nb_stop > 0: factorise the block rows k_first .. nb_stop - 1 only (see the kernel for what row_limit selects;
+// row_limit <= 0: all rows below are updated).  A partial run that updates everything below must not ask for Wm.
 inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* bar, int32_t* status,
-                          cudaStream_t stream, int nb_stop = 0) {
-    if (nb_stop > 0 && Wm != nullptr) return PTQ_ERR_INVALID_ARG;
-    if (nb_stop <= 0) nb_stop = (n + kNB - 1) / kNB;
+                          cudaStream_t stream, int nb_stop = 0, int k_first = 0, int row_limit = 0) {
+    const int nb_all = (n + kNB - 1) / kNB;
+    if (nb_stop <= 0) nb_stop = nb_all;
+    if (row_limit <= 0) row_limit = nb_all;
+    if (nb_stop < nb_all && row_limit > nb_stop && Wm != nullptr) return PTQ_ERR_INVALID_ARG;
+    if (k_first < 0 || k_first >= nb_stop) return PTQ_ERR_INVALID_ARG;
     DeviceState* dev = nullptr;
     int st = current_device_state(&dev);
     if (st) return st;
@@ -718,7 +728,7 @@ inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* 
     int64_t ld = n;
     int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;
     long long spin_limit = kSpinLimitCycles;
-    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status, &spin_limit, &nb_stop};
+    void* args[] = {&A, &Wm, &Dbuf, &n, &ld, &vec16, &bar, &status, &spin_limit, &k_first, &nb_stop, &row_limit};
     Launch l(K_CHOL_COOP, stream);
     if (cudaLaunchCooperativeKernel((const void*)chol_coop_kernel, dim3(grid), dim3(kCholThreads), args,
                                     kCholSmemBytes, stream) != cudaSuccess) {

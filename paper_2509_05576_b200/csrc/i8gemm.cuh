@@ -164,7 +164,8 @@ __global__ void __launch_bounds__(256) x_slice_cols_kernel(const double* __restr
 }
 
 // Output modes: what the epilogue does with P = A B^T.
-enum { X_OUT_ADD = 0,        // C += alpha P
+enum { X_OUT_ADD_UPPER = 3,  // C += alpha P on the tiles that touch the upper triangle only (A = B, C symmetric, upper kept)
+       X_OUT_ADD = 0,        // C += alpha P
        X_OUT_SYM = 1,        // C = alpha P on the tiles that touch the upper triangle, and C[j][i] = C[i][j] (A = B)
        X_OUT_REDUCE = 2 };   // partials[tile] = alpha * sum_ij P_ij D_ij ; C is not touched
 // K ranges per tile (operands known to be zero outside them, or terms accounted for elsewhere).
@@ -191,7 +192,7 @@ __device__ __forceinline__ bool x_tile_range(const XGemmParams& prm, int bi, int
     const int i0 = bi * kXTM, j0 = bj * kXTN;
     kb0 = 0;
     kb1 = nkb;
-    if (prm.out_mode == X_OUT_SYM && i0 > j0 + kXTN - 1) return false;
+    if ((prm.out_mode == X_OUT_SYM || prm.out_mode == X_OUT_ADD_UPPER) && i0 > j0 + kXTN - 1) return false;
     if (prm.k_mode == X_K_FROM_MAX) kb0 = (i0 > j0 ? i0 : j0) / kXKB;
     else if (prm.k_mode == X_K_BEFORE_J) kb1 = j0 / kXKB;
     else if (prm.k_mode == X_K_OWN_J) { kb0 = j0 / kXKB; kb1 = kb0 + 1; }
@@ -420,15 +421,18 @@ i8gemm_kernel(const __grid_constant__ CUtensorMap tmapA, const __grid_constant__
                 const int col = col0 + ocol;
                 if (col < prm.n) {
                     const double fj = __longlong_as_double((long long)(1023 + 24 - prm.sh_b[col]) << 52);
-#pragma unroll 4
-                    for (int rr = 0; rr < 32; rr += 2) {
-                        const int grow = bi * kXTM + quarter * 32 + rr + orow;
-                        if (grow < prm.m) {
-                            double* dst = prm.C + (int64_t)grow * prm.ldc + col;
-                            const double pv = my[(rr + orow) * 17 + ocol] * fj;
-                            *dst = prm.out_mode == X_OUT_ADD ? *dst + pv : pv;
-                        }
-                    }
+                    double* dst0 = prm.C + (int64_t)(bi * kXTM + quarter * 32 + orow) * prm.ldc + col;
+                    const int rows_left = prm.m - (bi * kXTM + quarter * 32 + orow);      // rows rr with rr < rows_left exist
+                    // all sixteen old values are requested before the first is used: one memory latency per chunk
+                    double oldv[16];
+#pragma unroll
+                    for (int q = 0; q < 16; ++q)
+                        oldv[q] = (prm.out_mode != X_OUT_SYM && 2 * q < rows_left)
+                                      ? __ldcg(dst0 + (int64_t)(2 * q) * prm.ldc) : 0.0;
+#pragma unroll
+                    for (int q = 0; q < 16; ++q)
+                        if (2 * q < rows_left)
+                            __stcg(dst0 + (int64_t)(2 * q) * prm.ldc, oldv[q] + my[(2 * q + orow) * 17 + ocol] * fj);
                 }
                 __syncwarp();
             }
