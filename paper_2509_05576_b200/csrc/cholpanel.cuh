@@ -3,7 +3,7 @@
 // 64 kPanelBlocks on the int8 tensor path (i8gemm.cuh),
 //     A[i][j] -= sum_{r in panel} U[r][i] U[r][j]   (i, j below the panel, upper tiles),
 //     W[i][c] -= sum_{r in panel} U[r][i] W[r][c]   (i below the panel, c up to its end),
-// instead of one 64-deep float64 MMA update per block row: with a depth of 512 the product moves a fifth of the bytes
+// instead of one 64-deep float64 MMA update per block row: with a depth of 1024 the product moves a small fraction of the bytes
 // per multiply-add through L2.  The blocked form of Eq. 12 / Sec. 5 item 1 is unchanged, only the grouping of the updates.
 #pragma once
 #include "chol.cuh"
@@ -11,7 +11,7 @@
 
 namespace ptq {
 
-constexpr int kPanelBlocks = 8;              // 512 columns per panel
+constexpr int kPanelBlocks = 16;             // 1024 columns per panel
 constexpr int kPanelMinCols = 3072;          // below this the single cooperative launch is faster
 
 inline size_t chol_panel_workspace_bytes(int n) {
