@@ -40,7 +40,7 @@ inline size_t i8gemm_plane_bytes(int rows, int k) {
 }
 inline size_t i8gemm_workspace_bytes(int m, int n, int k) {
     return align_up(i8gemm_plane_bytes(m, k)) + align_up(i8gemm_plane_bytes(n, k)) +
-           align_up((size_t)(cdiv(m, 128) * 128) * sizeof(int32_t)) + align_up((size_t)(cdiv(n, 128) * 128) * sizeof(int32_t));
+           align_up((size_t)(cdiv(m, 128) * 128) * 12) + align_up((size_t)(cdiv(n, 128) * 128) * 12) + 1024;
 }
 // Output / K-range modes and the slicing of one operand at a time: see XGemmParams, x_slice_operand, x_product below.
 
@@ -107,36 +107,50 @@ __global__ void __launch_bounds__(256) x_slice_rows_kernel(const double* __restr
 }
 
 // Slices of the COLUMNS of X [k x cols] (row stride ld): Q[s][col][kk] -- the operand B of C += A B^T when the matrix
-// at hand is stored as [k][j].  One CTA per 32 columns: column maxima first (reads along rows are coalesced), then
-// 32 x 32 tiles are read row-wise, cut into digits and written out transposed through shared memory.
-__global__ void __launch_bounds__(256) x_slice_cols_kernel(const double* __restrict__ X, int k, int cols, int64_t ld,
-                                                            int cols_pad, int k_pad, int8_t* __restrict__ Q,
-                                                            int32_t* __restrict__ shifts) {
+// at hand is stored as [k][j].  Two passes, both over a grid of (32-column groups) x (256-row chunks of k), so that a
+// deep operand is spread over many CTAs: x_colmax_kernel takes the column maxima (reads along rows are coalesced; the
+// maxima of the chunks meet by an integer atomic maximum on the bit patterns, which orders non-negative doubles as it
+// orders integers and does not depend on the order of arrival); x_slice_cols_kernel reads 32 x 32 tiles row-wise, cuts
+// them into digits and writes them out transposed through shared memory.
+constexpr int kXColChunk = 256;
+__global__ void __launch_bounds__(256) x_colmax_kernel(const double* __restrict__ X, int k, int cols, int64_t ld,
+                                                        unsigned long long* __restrict__ colmax) {
     __shared__ double smax[8][33];
-    __shared__ int ssh[32];
+    const int c0 = blockIdx.x * 32, k0 = blockIdx.y * kXColChunk;
+    const int lane = threadIdx.x & 31, wy = threadIdx.x >> 5;
+    const int col = c0 + lane;
+    const int k1 = k0 + kXColChunk < k ? k0 + kXColChunk : k;
+    double m = 0.0;
+    if (col < cols)
+        for (int kk = k0 + wy; kk < k1; kk += 8) {
+            const double a = fabs(X[(int64_t)kk * ld + col]);
+            m = a > m || !(a == a) ? a : m;                   // a NaN sticks, so that the column is treated as dead
+        }
+    smax[wy][lane] = m;
+    __syncthreads();
+    if (wy == 0 && col < cols) {
+        double mm = smax[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) mm = (smax[w][lane] > mm || !(smax[w][lane] == smax[w][lane])) ? smax[w][lane] : mm;
+        // NaN and infinity have bit patterns above every finite double: they win the maximum as well
+        atomicMax(colmax + col, (unsigned long long)__double_as_longlong(mm));
+    }
+}
+__global__ void __launch_bounds__(256) x_slice_cols_kernel(const double* __restrict__ X, int k, int cols, int64_t ld,
+                                                            int cols_pad, int k_pad,
+                                                            const unsigned long long* __restrict__ colmax,
+                                                            int8_t* __restrict__ Q, int32_t* __restrict__ shifts) {
     __shared__ uint8_t dig[kXSlices][32][36];          // [slice][column][kk within the tile]
-    const int c0 = blockIdx.x * 32;
+    const int c0 = blockIdx.x * 32, kbeg = blockIdx.y * kXColChunk;
     const int lane = threadIdx.x & 31, wy = threadIdx.x >> 5;          // 8 row slices x 32 columns
     const size_t plane = (size_t)cols_pad * k_pad;
     const int col = c0 + lane;
-    double m = 0.0;
-    if (col < cols)
-        for (int kk = wy; kk < k; kk += 8) m = fmax(m, fabs(X[(int64_t)kk * ld + col]));
-    smax[wy][lane] = m;
-    __syncthreads();
-    if (wy == 0) {
-        double mm = smax[0][lane];
-#pragma unroll
-        for (int w = 1; w < 8; ++w) mm = fmax(mm, smax[w][lane]);
-        const int sh = x_row_shift(mm);
-        ssh[lane] = (mm > 0.0 && mm < 1.0e300) ? sh : (1 << 30);          // 1 << 30: dead column
-        if (c0 + lane < cols_pad) shifts[c0 + lane] = (mm > 0.0 && mm < 1.0e300) ? sh : 0;
-    }
-    __syncthreads();
-    const int sh_raw = ssh[lane];
-    const bool dead = sh_raw == (1 << 30) || col >= cols;
-    const int sh = dead ? 0 : sh_raw;
-    for (int k0 = 0; k0 < k_pad; k0 += 32) {
+    const double mm = col < cols ? __longlong_as_double((long long)colmax[col]) : 0.0;
+    const bool dead = !(mm > 0.0 && mm < 1.0e300);
+    const int sh = dead ? 0 : x_row_shift(mm);
+    if (blockIdx.y == 0 && wy == 0 && col < cols_pad) shifts[col] = sh;
+    const int kend = kbeg + kXColChunk < k_pad ? kbeg + kXColChunk : k_pad;
+    for (int k0 = kbeg; k0 < kend; k0 += 32) {
         // thread (wy, lane): rows k0 + wy, + 8, + 16, + 24 of column `col`
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
@@ -471,7 +485,8 @@ struct XOperand {
     int rows, k;
 };
 inline size_t x_operand_bytes(int rows, int k) {
-    return align_up(i8gemm_plane_bytes(rows, k)) + align_up((size_t)(cdiv(rows, 128) * 128) * sizeof(int32_t));
+    return align_up(i8gemm_plane_bytes(rows, k)) + align_up((size_t)(cdiv(rows, 128) * 128) * sizeof(int32_t)) +
+           align_up((size_t)(cdiv(rows, 128) * 128) * sizeof(unsigned long long));
 }
 // X is [rows x k] (transposed = 0, row stride ld) or [k x rows] (transposed = 1: the operand's rows are X's columns).
 inline XOperand x_slice_operand(Carver& cv, const double* X, int64_t ld, int transposed, int rows, int k,
@@ -480,12 +495,17 @@ inline XOperand x_slice_operand(Carver& cv, const double* X, int64_t ld, int tra
     XOperand op;
     op.Q = cv.take<int8_t>(i8gemm_plane_bytes(rows, k));
     op.sh = cv.take<int32_t>(rows_pad);
+    unsigned long long* colmax = cv.take<unsigned long long>(rows_pad);
     op.rows = rows; op.k = k;
     Launch l(K_X_SLICE, stream);
-    if (transposed)
-        x_slice_cols_kernel<<<rows_pad / 32, 256, 0, stream>>>(X, k, rows, ld, rows_pad, k_pad, op.Q, op.sh);
-    else
+    if (transposed) {
+        cudaMemsetAsync(colmax, 0, (size_t)rows_pad * sizeof(unsigned long long), stream);
+        x_colmax_kernel<<<dim3(rows_pad / 32, cdiv(k, kXColChunk)), 256, 0, stream>>>(X, k, rows, ld, colmax);
+        x_slice_cols_kernel<<<dim3(rows_pad / 32, cdiv(k_pad, kXColChunk)), 256, 0, stream>>>(X, k, rows, ld, rows_pad, k_pad,
+                                                                                              colmax, op.Q, op.sh);
+    } else {
         x_slice_rows_kernel<<<rows_pad, 256, 0, stream>>>(X, rows, k, ld, rows_pad, k_pad, op.Q, op.sh);
+    }
     return op;
 }
 
