@@ -125,37 +125,47 @@ __device__ __forceinline__ unsigned long long sortable_key(double x) {
 
 // perm[rank_j] = j with rank_j = #{k : S_k > S_j, or S_k == S_j and k < j}: a stable descending sort by counting
 // (ascending != 0: S_k < S_j instead, the "asc" keys of Sec. 4.1; equal scores keep the lower index first either way).
-// 32 columns j per CTA; the eight lanes that share a column each count a strided eighth of the keys.
-constexpr int kRankCols = 32;
+// 16 columns j per CTA; the 16 lanes that share a column each count a strided sixteenth of the keys, which are staged in
+// shared memory 2048 at a time.  A chunk is padded to a multiple of 128 keys with entries that never count (key 0 with
+// the largest tie value), so the counting loop runs in unrolled groups of eight without a bound test.
+constexpr int kRankCols = 16;
+constexpr int kRankChunk = 2048;
 // tie != nullptr: equal scores are ordered by tie[] (distinct values) instead of by position.
 __global__ void __launch_bounds__(256) rank_sort_kernel(const double* __restrict__ S, int cols, int ascending,
                                                          int32_t* __restrict__ perm,
                                                          const int32_t* __restrict__ tie = nullptr) {
-    __shared__ unsigned long long keys[1024];
-    __shared__ int32_t ties[1024];
-    const int j = blockIdx.x * kRankCols + (threadIdx.x >> 3);
-    const int part = threadIdx.x & 7;
+    __shared__ unsigned long long keys[kRankChunk];
+    __shared__ int32_t ties[kRankChunk];
+    const int j = blockIdx.x * kRankCols + (threadIdx.x >> 4);
+    const int part = threadIdx.x & 15;
     // ascending order is descending order of the complemented keys
     const unsigned long long flip = ascending ? ~0ull : 0ull;
     const unsigned long long kj = j < cols ? (sortable_key(S[j]) ^ flip) : 0ull;
     const int tj = (tie != nullptr && j < cols) ? tie[j] : j;
     int rank = 0;
-    for (int t0 = 0; t0 < cols; t0 += 1024) {
-        for (int t = threadIdx.x; t < 1024; t += 256) {
-            keys[t] = t0 + t < cols ? (sortable_key(S[t0 + t]) ^ flip) : 0ull;
-            ties[t] = (tie != nullptr && t0 + t < cols) ? tie[t0 + t] : t0 + t;
+    for (int t0 = 0; t0 < cols; t0 += kRankChunk) {
+        const int lim = min(kRankChunk, cols - t0);
+        const int lim_pad = (lim + 127) & ~127;
+        for (int t = threadIdx.x; t < lim_pad; t += 256) {
+            const bool in = t < lim;
+            keys[t] = in ? (sortable_key(S[t0 + t]) ^ flip) : 0ull;
+            ties[t] = in ? (tie != nullptr ? tie[t0 + t] : t0 + t) : 0x7fffffff;
         }
         __syncthreads();
-        const int lim = min(1024, cols - t0);
-        for (int t = part; t < lim; t += 8) {
-            const unsigned long long kk = keys[t];
-            rank += (kk > kj || (kk == kj && ties[t] < tj)) ? 1 : 0;
+        for (int base = part; base < lim_pad; base += 128) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const unsigned long long kk = keys[base + 16 * u];
+                const int tt = ties[base + 16 * u];
+                rank += (kk > kj || (kk == kj && tt < tj)) ? 1 : 0;
+            }
         }
         __syncthreads();
     }
     rank += __shfl_xor_sync(0xffffffffu, rank, 1);
     rank += __shfl_xor_sync(0xffffffffu, rank, 2);
     rank += __shfl_xor_sync(0xffffffffu, rank, 4);
+    rank += __shfl_xor_sync(0xffffffffu, rank, 8);
     if (part == 0 && j < cols) perm[rank] = j;
 }
 
