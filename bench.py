@@ -205,6 +205,7 @@ def layer_set_totals(fp64_peak, flush, ws):
     """The configurations beyond the single bench layer, measured in this run: the ResNet-50-shaped set (4-bit), the
     YOLOv5s-shaped set (8- and 4-bit) and the scaling shapes at 3, 4 and 8 bits.  Per set: total ms, weights/s, per-stage
     ms and per-stage roofline fraction (sum of algorithmic work / sum of stage time / peak)."""
+    import torch
     from paper_2509_05576_b200 import layer_set_run as lsr
 
     def brief(res, per_layer=False):
@@ -216,8 +217,8 @@ def layer_set_totals(fp64_peak, flush, ws):
         return out
 
     sets = {}
-    sets["c3_resnet50_w4"] = brief(lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True),
-                                   per_layer=True)
+    res3 = lsr.run_specs(wl.config3(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True)
+    sets["c3_resnet50_w4"] = brief(res3, per_layer=True)
     # the YOLOv5s-shaped layers at 8 and 4 bits share their inputs: run the two bit-widths of a layer back to back
     c4 = [s for pair in zip(wl.config4(bits=(8,)), wl.config4(bits=(4,))) for s in pair]
     res4 = lsr.run_specs(c4, 2, fp64_peak=fp64_peak, ws=ws, flush=flush, graphs=True)
@@ -233,11 +234,22 @@ def layer_set_totals(fp64_peak, flush, ws):
                                     "weights_per_s": wts / (ms * 1e-3),
                                     "graph_total_ms": sum(r["graph_ms"] for r in rows), "stage_total_ms": st}
     sets["c4_yolov5s_w8"]["stage_roofline_frac_both_bit_widths"] = res4["stage_roofline_frac"]
-    # independent layers of a set overlapped on four streams (the small layers leave most SMs idle on their own)
-    sets["c3_resnet50_w4"]["overlapped_4_streams_ms"] = lsr.run_overlapped(wl.config3(), 4, 2, flush=flush)["set_ms"]
+    # Independent layers of a set overlapped on streams (the small layers leave most SMs idle on their own): four
+    # streams as they come, and eight streams with the persistent cooperative kernels held to a quarter of the SMs each
+    # (half for the wide layers), layers dealt longest first.  Same results either way (the sum of the losses is checked).
+    def overlapped(specs, ref_loss):
+        a4 = lsr.run_overlapped(specs, 4, 2, flush=flush)
+        sms = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+        a8 = lsr.run_overlapped(specs, 8, 2, flush=flush, cta_limit=max(1, sms // 4))
+        for a in (a4, a8):
+            if abs(a["loss_sum"] - ref_loss) > 1e-9 * abs(ref_loss):
+                raise RuntimeError("overlapped layer set: the losses differ from the one-stream run")
+        return {"overlapped_4_streams_ms": a4["set_ms"], "overlapped_8_streams_cta_limited_ms": a8["set_ms"],
+                "weights_per_s_overlapped": sum(sp.rows * sp.cols for sp in specs) / (a8["set_ms"] * 1e-3)}
+    sets["c3_resnet50_w4"].update(overlapped(wl.config3(), sum(r["loss"] for r in res3["layers"])))
     for b in (8, 4):
-        sets[f"c4_yolov5s_w{b}"]["overlapped_4_streams_ms"] = lsr.run_overlapped(wl.config4(bits=(b,)), 4, 2,
-                                                                                 flush=flush)["set_ms"]
+        sets[f"c4_yolov5s_w{b}"].update(overlapped(wl.config4(bits=(b,)),
+                                                   sum(r["loss"] for r in res4["layers"] if r["bits"] == b)))
     sets["c5_scaling_w3_w4_w8"] = brief(lsr.run_specs(wl.config5(), 2, fp64_peak=fp64_peak, ws=ws, flush=flush),
                                         per_layer=True)
     return sets

@@ -268,6 +268,14 @@ int ptq_fp64_probe(int kind, int iters, double *sink, double *flops_out, void *s
  *   ptq_profile_read(id, total_ms, launches) : host pointers; waits for the recorded events and sums the device
  *                            time of kernel `id` over the recorded launches.
  */
+/* The two persistent cooperative kernels (factorisation, column sweep) launch one CTA per SM and occupy an SM each, so
+ * two of them never share the GPU.  ptq_set_cta_limit(limit) makes the calls issued afterwards ON THE CURRENT DEVICE
+ * launch at most `limit` CTAs (0: no limit, the default): a caller that runs independent layers on several streams sets
+ * about sm_count / streams, so that their factorisations and sweeps run side by side (those of layers up to a few thousand
+ * columns are bound by a dependency chain, not by the number of SMs).  Results do not depend on the limit.
+ * Returns PTQ_ERR_INVALID_ARG for a negative limit. */
+int ptq_set_cta_limit(int limit);
+
 int ptq_kernel_count(void);
 const char *ptq_kernel_name(int kernel_id);
 long long ptq_launch_count(int kernel_id);

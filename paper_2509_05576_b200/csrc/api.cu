@@ -146,6 +146,16 @@ long long ptq_launch_count(int kernel_id) {
     return total;
 }
 
+int ptq_set_cta_limit(int limit) {
+    if (limit < 0) return PTQ_ERR_INVALID_ARG;
+    DeviceState* dev = nullptr;
+    const int st = current_device_state(&dev);
+    if (st) return st;
+    std::lock_guard<std::mutex> lock(host_state_mutex());
+    dev->cta_limit = limit;
+    return PTQ_OK;
+}
+
 int ptq_profile_enable(int on) {
     Profiler& p = profiler();
     p.clear();

@@ -723,7 +723,8 @@ inline int cholesky_upper(double* A, int n, double* Wm, double* Dbuf, unsigned* 
     // of other streams.
     const int nbr = (n + kNB - 1) / kNB;
     const long items = (long)nbr * (nbr + 1) / 2 + (Wm != nullptr ? (long)nbr * nbr : 0);
-    const int grid = items < dev->sms ? (int)(items < 1 ? 1 : items) : dev->sms;
+    const int budget = coop_cta_budget(dev);
+    const int grid = items < budget ? (int)(items < 1 ? 1 : items) : budget;
     if (cudaMemsetAsync(bar, 0, 2 * sizeof(unsigned), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int64_t ld = n;
     int vec16 = ((n & 1) == 0 && aligned16(A) && aligned16(Wm)) ? 1 : 0;

@@ -567,7 +567,7 @@ inline int sweep_launch(double* Wp, const double* U, double* E, uint8_t* codes_p
     if (st) return st;
     // one CTA per SM; with few row groups only the CTAs that get a share of the blocks are launched
     const int groups_l = cdiv(rows, kSweepRows), nb_l = cdiv(n, kNB);
-    int grid = dev->sms;
+    int grid = coop_cta_budget(dev);
     if (groups_l < grid) {
         const int per = grid / groups_l < nb_l ? grid / groups_l : nb_l;
         grid = groups_l * per;

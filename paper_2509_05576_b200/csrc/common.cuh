@@ -96,6 +96,7 @@ enum SmemAttrSlot { SA_CHOL = 0, SA_SWEEP, SA_GRAM, SA_DGEMM, SA_SMALL, SA_XGEMM
 struct DeviceState {
     int sms = 0;
     int coop = 0;
+    int cta_limit = 0;            // > 0: the persistent cooperative kernels launch at most this many CTAs (ptq_set_cta_limit)
     bool attr[SA_COUNT] = {};
 };
 inline std::mutex& host_state_mutex() { static std::mutex mu; return mu; }
@@ -114,6 +115,11 @@ inline int current_device_state(DeviceState** out) {
     }
     *out = &d;
     return PTQ_OK;
+}
+// CTAs a persistent cooperative kernel may launch on this device: one per SM, or the caller's limit if that is lower.
+inline int coop_cta_budget(const DeviceState* d) {
+    std::lock_guard<std::mutex> lock(host_state_mutex());
+    return (d->cta_limit > 0 && d->cta_limit < d->sms) ? d->cta_limit : d->sms;
 }
 // Runs `set` (the cudaFuncSetAttribute calls of one kernel family) once per device.
 template <typename F>

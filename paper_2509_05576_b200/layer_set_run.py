@@ -162,10 +162,16 @@ def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP
             "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak, "fp64_tflops": fp64_peak, "source": src}}
 
 
-def run_overlapped(specs, n_streams, reps=2, score_mode=ptq.SCORE_QERR, flush=None):
+BIG_FACTOR = 2.0
+
+
+def run_overlapped(specs, n_streams, reps=2, score_mode=ptq.SCORE_QERR, flush=None, cta_limit=0):
     """The whole set with independent layers dealt round-robin onto `n_streams` streams: every stream has its own
     workspace, every layer its own output buffers, the inputs of all layers are put on the device first, one event pair
-    around the whole set (median of `reps` timed passes after one warm-up pass)."""
+    around the whole set (median of `reps` timed passes after one warm-up pass).  cta_limit > 0: the persistent
+    cooperative kernels of layers below 3072 columns (bound by their dependency chains, not by the SM count) launch at
+    most that many CTAs each, so that those of different streams run side by side; the layers are then also dealt
+    longest first onto the stream with the least work so far (estimated from the shapes)."""
     s = torch.cuda.current_stream()
     flush = flush if flush is not None else torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
     data = []
@@ -176,9 +182,21 @@ def run_overlapped(specs, n_streams, reps=2, score_mode=ptq.SCORE_QERR, flush=No
     streams = [torch.cuda.Stream() for _ in range(n_streams)]
     wss = [ptq.Workspace() for _ in streams]
 
+    plan = [(i, i % len(streams)) for i in range(len(data))]
+    if cta_limit > 0:
+        # rough device time of a layer in ms: fixed part, the two chains per 64 columns, the cubic part
+        est = [0.1 + 0.04 * s_.cols / 64 + 6.0 * (s_.cols / 4608.0) ** 3 * (1 + s_.rows / 4096.0) for s_ in specs]
+        load = [0.0] * len(streams)
+        plan = []
+        for i in sorted(range(len(data)), key=lambda q: -est[q]):
+            k = min(range(len(streams)), key=lambda q: load[q])
+            load[k] += est[i]
+            plan.append((i, k))
+
     def run_set():
-        for i, (spec, Wd, Xd) in enumerate(data):
-            k = i % len(streams)
+        for i, k in plan:
+            spec, Wd, Xd = data[i]
+            ptq.set_cta_limit(cta_limit if spec.cols < 3072 else int(cta_limit * BIG_FACTOR))
             ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=score_mode,
                                     bufs=outs[i], ws=wss[k], stream=streams[k])
 
@@ -197,9 +215,10 @@ def run_overlapped(specs, n_streams, reps=2, score_mode=ptq.SCORE_QERR, flush=No
         torch.cuda.synchronize()
         if rep > 0:
             times.append(e0.elapsed_time(e1))
+    ptq.set_cta_limit(0)
     for o, spec in zip(outs, specs):
         ptq.check_status(o.status, spec.name)
-    return {"streams": n_streams, "set_ms": float(np.median(times)),
+    return {"streams": n_streams, "cta_limit": cta_limit, "set_ms": float(np.median(times)),
             "loss_sum": float(sum(o.loss.item() for o in outs))}
 
 
@@ -213,6 +232,8 @@ def main(argv=None):
     ap.add_argument("--streams", type=int, default=1,
                     help="> 1: also run the whole set with the layers dealt round-robin onto this many streams "
                          "(inputs resident, nothing synchronised in between) and report the wall time of that")
+    ap.add_argument("--cta-limit", type=int, default=0,
+                    help="with --streams: at most this many CTAs per persistent cooperative kernel (0: one per SM)")
     ap.add_argument("--score-mode", default="qerr", choices=sorted(SCORE_MODES),
                     help="column ordering: qerr (Eq. 10, the method's), prune (Eq. 8), err, w, none (no sorting)")
     ap.add_argument("--ascending", action="store_true", help="sort the scores ascending (the 'asc' keys of Sec. 4.1)")
@@ -239,7 +260,7 @@ def main(argv=None):
     totals = {"ms": res["total_ms"]}
     overlapped = None
     if args.streams > 1:
-        overlapped = run_overlapped(specs, args.streams, args.reps, mode, flush)
+        overlapped = run_overlapped(specs, args.streams, args.reps, mode, flush, args.cta_limit)
         print(f"whole set on {args.streams} streams: {overlapped['set_ms']:.2f} ms "
               f"(sum of the per-layer times on one stream: {totals['ms']:.2f} ms)")
     print(json.dumps({"config": args.config, "score_mode": args.score_mode, "ascending": bool(args.ascending),

@@ -28,7 +28,8 @@ CALL_QUANTIZE_LAYER_PER_ROW = 6
 EXPORTS = ["ptq_workspace_bytes", "ptq_hessian_accumulate", "ptq_hessian_accumulate_conv", "ptq_hessian_accumulate_f64", "ptq_prepare_hinv",
            "ptq_minmax_grid", "ptq_sensitivity_order", "ptq_sensitivity_order_static", "ptq_quantize_layer", "ptq_status_string", "ptq_version",
            "ptq_sort_scores", "ptq_gemm_nt_sliced", "ptq_gemm_nt_sliced_workspace_bytes", "ptq_quantize_layer_dynamic", "ptq_quantize_layer_per_row", "ptq_selftest_wait_timeout", "ptq_fp64_probe",
-           "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read"]
+           "ptq_kernel_count", "ptq_kernel_name", "ptq_launch_count", "ptq_profile_enable", "ptq_profile_read",
+           "ptq_set_cta_limit"]
 
 
 class PtqError(RuntimeError):
@@ -86,6 +87,7 @@ def lib():
         L.ptq_launch_count.argtypes = [c_int]
         L.ptq_launch_count.restype = ctypes.c_longlong
         L.ptq_profile_enable.argtypes = [c_int]
+        L.ptq_set_cta_limit.argtypes = [c_int]
         L.ptq_profile_read.argtypes = [c_int, ctypes.POINTER(c_double), ctypes.POINTER(ctypes.c_longlong)]
         _lib = L
     return _lib
@@ -98,6 +100,11 @@ def status_string(code: int) -> str:
 def launch_count(kernel_id: int = -1) -> int:
     """Kernel launches made by the library in this process (all kernels when kernel_id < 0)."""
     return int(lib().ptq_launch_count(int(kernel_id)))
+
+
+def set_cta_limit(limit: int):
+    """At most `limit` CTAs per persistent cooperative kernel on the current device (0: one per SM)."""
+    _check(lib().ptq_set_cta_limit(int(limit)), "ptq_set_cta_limit")
 
 
 def profile_enable(on: bool):

@@ -390,3 +390,22 @@ def test_layer_path_replayed_as_a_cuda_graph_matches_the_eager_path():
     ref = oracle_layer(W2, X2, 4)
     out = {k: getattr(bufs, k).cpu().numpy() for k in ("perm", "scale", "zero", "codes", "What", "loss")}
     assert assert_layer_parity(out, ref) == 0
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("rows,cols,limit", [(96, 700, 5), (300, 200, 3), (2500, 130, 20)])
+def test_cta_limit_changes_the_grids_not_the_results(rows, cols, limit):
+    """ptq_set_cta_limit holds the persistent cooperative kernels (factorisation, sweep) to a few CTAs; every array of the
+    layer's result is the same, bit for bit, as with one CTA per SM.  The shapes give fewer CTAs than block rows of the
+    factorisation, than row groups of the sweep, and fewer than either."""
+    W, X = _layer(rows, cols, 384, 4242)
+    g = gpu_layer(W, X, 4)
+    ptq.set_cta_limit(limit)
+    try:
+        h = gpu_layer(W, X, 4)
+    finally:
+        ptq.set_cta_limit(0)
+    for k in ("H", "Hinv", "S", "perm", "codes", "What", "loss"):
+        assert np.array_equal(h[k], g[k]), k
+    with pytest.raises(ptq.PtqError):
+        ptq.set_cta_limit(-1)
