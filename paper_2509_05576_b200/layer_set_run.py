@@ -162,60 +162,28 @@ def run_specs(specs, reps=2, score_mode=ptq.SCORE_QERR, quiet=True, fp64_peak=FP
             "peaks": {"hbm_gbs": hbm, "int8_tflops": int8_peak, "fp64_tflops": fp64_peak, "source": src}}
 
 
-BIG_FACTOR = 2.0
-
-
 def run_overlapped(specs, n_streams, reps=2, score_mode=ptq.SCORE_QERR, flush=None, cta_limit=0):
-    """The whole set with independent layers dealt round-robin onto `n_streams` streams: every stream has its own
-    workspace, every layer its own output buffers, the inputs of all layers are put on the device first, one event pair
-    around the whole set (median of `reps` timed passes after one warm-up pass).  cta_limit > 0: the persistent
-    cooperative kernels of layers below 3072 columns (bound by their dependency chains, not by the SM count) launch at
-    most that many CTAs each, so that those of different streams run side by side; the layers are then also dealt
-    longest first onto the stream with the least work so far (estimated from the shapes)."""
+    """The whole set through ``ptq.LayerSet``: independent layers side by side on `n_streams` streams, the inputs of all
+    layers put on the device first, one event pair around the whole set (median of `reps` timed passes after one warm-up
+    pass).  cta_limit 0: layers dealt round-robin, cooperative kernels with one CTA per SM; > 0: see ``ptq.LayerSet``."""
     s = torch.cuda.current_stream()
     flush = flush if flush is not None else torch.empty(256 * 2 ** 20, dtype=torch.uint8, device="cuda")
-    data = []
+    layers = []
     for spec in specs:
         W, X = wl.make_layer(spec)
-        data.append((spec, torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda()))
-    outs = [ptq.LayerBuffers(spec.rows, spec.cols) for spec in specs]      # one set of outputs per layer, kept
-    streams = [torch.cuda.Stream() for _ in range(n_streams)]
-    wss = [ptq.Workspace() for _ in streams]
-
-    plan = [(i, i % len(streams)) for i in range(len(data))]
-    if cta_limit > 0:
-        # rough device time of a layer in ms: fixed part, the two chains per 64 columns, the cubic part
-        est = [0.1 + 0.04 * s_.cols / 64 + 6.0 * (s_.cols / 4608.0) ** 3 * (1 + s_.rows / 4096.0) for s_ in specs]
-        load = [0.0] * len(streams)
-        plan = []
-        for i in sorted(range(len(data)), key=lambda q: -est[q]):
-            k = min(range(len(streams)), key=lambda q: load[q])
-            load[k] += est[i]
-            plan.append((i, k))
-
-    def run_set():
-        for i, k in plan:
-            spec, Wd, Xd = data[i]
-            ptq.set_cta_limit(cta_limit if spec.cols < 3072 else int(cta_limit * BIG_FACTOR))
-            ptq.quantize_layer_full(Wd, Xd, spec.bits, spec.damp, score_mode=score_mode,
-                                    bufs=outs[i], ws=wss[k], stream=streams[k])
-
+        layers.append((torch.from_numpy(W).cuda(), torch.from_numpy(X).cuda(), spec.bits, spec.damp))
+    ls = ptq.LayerSet(layers, n_streams, cta_limit, score_mode)
     times = []
     for rep in range(reps + 1):
         torch.cuda.synchronize()
         flush.fill_(rep)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(s)
-        for st_ in streams:
-            st_.wait_stream(s)
-        run_set()
-        for st_ in streams:
-            s.wait_stream(st_)
+        outs = ls.run()
         e1.record(s)
         torch.cuda.synchronize()
         if rep > 0:
             times.append(e0.elapsed_time(e1))
-    ptq.set_cta_limit(0)
     for o, spec in zip(outs, specs):
         ptq.check_status(o.status, spec.name)
     return {"streams": n_streams, "cta_limit": cta_limit, "set_ms": float(np.median(times)),

@@ -418,6 +418,58 @@ class LayerGraph:
         return self.bufs
 
 
+class LayerSet:
+    """Independent layers (a network's layers, each with its own calibration input) quantized side by side on several
+    streams of one GPU.  Layers up to a few thousand columns are bound by dependency chains (the pivots of the
+    factorisations, the columns of the sweep), not by the number of SMs, so several of them fit on the GPU at once --
+    provided the two persistent cooperative kernels, which otherwise take one CTA per SM each, are held to a share of the
+    SMs (``ptq_set_cta_limit``).  ``cta_limit`` None: a quarter of the SMs for layers below 3072 columns, half for wider
+    ones; 0: no limit.  The layers are dealt longest first (a rough estimate from the shapes) onto the stream with the
+    least work so far.  Every stream has its own workspace, every layer its own LayerBuffers, kept in ``self.bufs`` in
+    the order the layers were given; results do not depend on the placement.
+
+    ``layers``: list of (W, X, bits) or (W, X, bits, damp) with W [rows, cols] float32 and X [cols, n] float32 on the
+    device.  ``run()`` issues the whole set asynchronously (the streams first wait for the current stream, which in turn
+    waits for them at the end) and returns ``self.bufs``; synchronise and ``check_status`` before reading."""
+
+    def __init__(self, layers, n_streams=8, cta_limit=None, score_mode=SCORE_QERR, damp_mode=DAMP_REL_MEAN_DIAG):
+        self.layers = [tuple(l) if len(l) == 4 else (l[0], l[1], l[2], 0.01) for l in layers]
+        dev = self.layers[0][0].device
+        self.score_mode, self.damp_mode = score_mode, damp_mode
+        self.streams = [torch.cuda.Stream(device=dev) for _ in range(max(1, n_streams))]
+        self.wss = [Workspace(dev) for _ in self.streams]
+        self.bufs = [LayerBuffers(W.shape[0], W.shape[1], dev) for W, _, _, _ in self.layers]
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        self.cta_limit = max(1, sms // 4) if cta_limit is None else int(cta_limit)
+        self.plan = [(i, i % len(self.streams)) for i in range(len(self.layers))]
+        if self.cta_limit > 0:
+            # rough device time of a layer in ms: fixed part, the two chains per 64 columns, the cubic part
+            est = [0.1 + 0.04 * W.shape[1] / 64 + 6.0 * (W.shape[1] / 4608.0) ** 3 * (1 + W.shape[0] / 4096.0)
+                   for W, _, _, _ in self.layers]
+            load = [0.0] * len(self.streams)
+            self.plan = []
+            for i in sorted(range(len(self.layers)), key=lambda q: -est[q]):
+                k = min(range(len(self.streams)), key=lambda q: load[q])
+                load[k] += est[i]
+                self.plan.append((i, k))
+
+    def run(self):
+        cur = torch.cuda.current_stream()
+        for st_ in self.streams:
+            st_.wait_stream(cur)
+        try:
+            for i, k in self.plan:
+                W, X, bits, damp = self.layers[i]
+                set_cta_limit(self.cta_limit if W.shape[1] < 3072 else 2 * self.cta_limit)
+                quantize_layer_full(W, X, bits, damp, self.damp_mode, self.score_mode, bufs=self.bufs[i], ws=self.wss[k],
+                                    stream=self.streams[k])
+        finally:
+            set_cta_limit(0)
+        for st_ in self.streams:
+            cur.wait_stream(st_)
+        return self.bufs
+
+
 class HostStaging:
     """Device landing buffers and the copy stream used by ``quantize_layer_from_host`` (allocated once per shape)."""
 

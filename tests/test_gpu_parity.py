@@ -409,3 +409,22 @@ def test_cta_limit_changes_the_grids_not_the_results(rows, cols, limit):
         assert np.array_equal(h[k], g[k]), k
     with pytest.raises(ptq.PtqError):
         ptq.set_cta_limit(-1)
+
+
+@pytest.mark.gpu
+def test_layer_set_on_several_streams_equals_the_layers_one_by_one():
+    """ptq.LayerSet: independent layers side by side on three streams with limited cooperative grids; every layer's
+    arrays are the same, bit for bit, as from its own call, whatever stream it landed on, and a second run of the same
+    set object gives them again."""
+    shapes = [(40, 300, 256, 4), (130, 64, 200, 3), (64, 520, 600, 8), (33, 147, 147, 4), (256, 128, 512, 4)]
+    data = [_layer(r, c, n, 900 + i, bits=b) for i, (r, c, n, b) in enumerate(shapes)]
+    single = [gpu_layer(W, X, b) for (W, X), (_, _, _, b) in zip(data, shapes)]
+    ls = ptq.LayerSet([(_cuda(W), _cuda(X), b) for (W, X), (_, _, _, b) in zip(data, shapes)], n_streams=3, cta_limit=7)
+    assert sorted(i for i, _ in ls.plan) == list(range(len(shapes)))
+    for _ in range(2):
+        outs = ls.run()
+        torch.cuda.synchronize()
+        for o, g in zip(outs, single):
+            ptq.check_status(o.status, "layer set")
+            for k in ("H", "Hinv", "S", "perm", "codes", "What", "loss"):
+                assert np.array_equal(getattr(o, k).cpu().numpy(), g[k]), k
