@@ -39,10 +39,10 @@ INT8_OVER_BF16 = 2.0                                   # nominal dense 4.5 / 2.2
 # profiles/, on the bench workload (Gram: scaled from the 16384-column capture by the calibration columns processed).
 # Each entry names the kernel sources it was taken with; when they have changed since, the traffic is reported as null.
 NCU_TRAFFIC = {
-    "chol_coop": {"bytes_per_launch": (42.38e6 + 4.18e6 + 21.73e6 + 0.43e6) / 2, "sources": ["chol.cuh", "dgemm.cuh"],
-                  "sha256_16": "ba808a6277b0347b"},
-    "sweep_coop": {"bytes_per_launch": 29.82e6 + 0.04e6, "sources": ["colloop.cuh"], "sha256_16": "0970e32c809f2ad1"},
-    "gram_i8_tcgen05": {"bytes_per_launch": (508.2e6 + 31.9e6) * 4096 / 16384, "sources": ["gram.cuh"],
+    "chol_coop": {"bytes_per_launch": (42.38e6 + 3.67e6 + 21.73e6 + 0.44e6) / 2, "sources": ["chol.cuh", "dgemm.cuh"],
+                  "sha256_16": "9c632fdcdf2fe5a3"},
+    "sweep_coop": {"bytes_per_launch": 29.93e6 + 0.05e6, "sources": ["colloop.cuh"], "sha256_16": "fe83446e7e43c9ac"},
+    "gram_i8_tcgen05": {"bytes_per_launch": (508.4e6 + 31.9e6) * 4096 / 16384, "sources": ["gram.cuh"],
                         "sha256_16": "67013082159ad65c"},
 }
 
