@@ -27,12 +27,14 @@ __global__ void perm_check_kernel(const int32_t* __restrict__ perm, int cols, in
 
 __device__ __forceinline__ int clamp_index(int j, int n) { return j < 0 ? 0 : (j >= n ? n - 1 : j); }
 
-// A[a][b] = Hinv[perm[a]][perm[b]]
+// A[a][b] = Hinv[perm[a]][perm[b]] for b from the start of row a's 64-column diagonal tile on: the factorisation and
+// everything after it read the upper triangle only (whole 64 x 64 tiles on the diagonal), the rest of A is left alone.
 __global__ void gather_sym_kernel(const double* __restrict__ Hinv, const int32_t* __restrict__ perm, int n,
                                   double* __restrict__ A) {
     const int a = blockIdx.y;
+    const int b_first = a & ~(kNB - 1);
     const int64_t src = (int64_t)clamp_index(perm[a], n) * n;
-    for (int b = blockIdx.x * blockDim.x + threadIdx.x; b < n; b += gridDim.x * blockDim.x)
+    for (int b = b_first + blockIdx.x * blockDim.x + threadIdx.x; b < n; b += gridDim.x * blockDim.x)
         A[(int64_t)a * n + b] = Hinv[src + clamp_index(perm[b], n)];
 }
 

@@ -418,6 +418,29 @@ class LayerGraph:
         return self.bufs
 
 
+def estimate_layer_ms(rows, cols):
+    """Rough device time of one layer in ms (fixed part, the two pivot chains per 64 columns, the cubic part), used only
+    to deal the layers of a set onto streams."""
+    return 0.1 + 0.04 * cols / 64 + 6.0 * (cols / 4608.0) ** 3 * (1 + rows / 4096.0)
+
+
+def plan_layer_set(shapes, n_streams, longest_first=True):
+    """[(layer index, stream index)] in issue order for layers of the given (rows, cols).  longest_first: the layers in
+    descending order of their estimated time, each onto the stream with the least estimated work so far (ties: the lower
+    stream index); otherwise round-robin in the given order."""
+    n_streams = max(1, int(n_streams))
+    if not longest_first:
+        return [(i, i % n_streams) for i in range(len(shapes))]
+    est = [estimate_layer_ms(r, c) for r, c in shapes]
+    load = [0.0] * n_streams
+    plan = []
+    for i in sorted(range(len(shapes)), key=lambda q: (-est[q], q)):
+        k = min(range(n_streams), key=lambda q: (load[q], q))
+        load[k] += est[i]
+        plan.append((i, k))
+    return plan
+
+
 class LayerSet:
     """Independent layers (a network's layers, each with its own calibration input) quantized side by side on several
     streams of one GPU.  Layers up to a few thousand columns are bound by dependency chains (the pivots of the
@@ -441,17 +464,8 @@ class LayerSet:
         self.bufs = [LayerBuffers(W.shape[0], W.shape[1], dev) for W, _, _, _ in self.layers]
         sms = torch.cuda.get_device_properties(dev).multi_processor_count
         self.cta_limit = max(1, sms // 4) if cta_limit is None else int(cta_limit)
-        self.plan = [(i, i % len(self.streams)) for i in range(len(self.layers))]
-        if self.cta_limit > 0:
-            # rough device time of a layer in ms: fixed part, the two chains per 64 columns, the cubic part
-            est = [0.1 + 0.04 * W.shape[1] / 64 + 6.0 * (W.shape[1] / 4608.0) ** 3 * (1 + W.shape[0] / 4096.0)
-                   for W, _, _, _ in self.layers]
-            load = [0.0] * len(self.streams)
-            self.plan = []
-            for i in sorted(range(len(self.layers)), key=lambda q: -est[q]):
-                k = min(range(len(self.streams)), key=lambda q: load[q])
-                load[k] += est[i]
-                self.plan.append((i, k))
+        self.plan = plan_layer_set([tuple(W.shape) for W, _, _, _ in self.layers], len(self.streams),
+                                   longest_first=self.cta_limit > 0)
 
     def run(self):
         cur = torch.cuda.current_stream()

@@ -138,3 +138,26 @@ def test_conv_entry_point_rejects_bad_arguments_without_a_gpu(lib):
     assert f(None, fake, 1, 3, 8, 8, 3, 3, 1, 1, fake, 1 << 30, fake, None) == ptq.ERR_INVALID_ARG
     assert f(fake, fake, 1, 3, 8, 8, 3, 3, 1, 1, fake, 16, fake, None) == ptq.ERR_WORKSPACE
     assert f(fake, fake, 1, 1 << 18, 8, 8, 3, 3, 1, 1, fake, 1 << 40, fake, None) == ptq.ERR_UNSUPPORTED   # cols > 2^20
+
+
+def test_layer_set_plan_deals_every_layer_once_and_balances_the_streams():
+    """Host logic of ptq.LayerSet: the plan is a permutation of the layers, the longest layers are issued first, no
+    stream's estimated load exceeds the mean by more than the longest layer, and round-robin is kept when asked for."""
+    from paper_2509_05576_b200 import ptq
+    from paper_2509_05576_b200 import workloads as wl
+    shapes = [(s.rows, s.cols) for s in wl.config3()]
+    for n_streams in (1, 3, 8):
+        plan = ptq.plan_layer_set(shapes, n_streams)
+        assert sorted(i for i, _ in plan) == list(range(len(shapes)))
+        assert all(0 <= k < n_streams for _, k in plan)
+        est = [ptq.estimate_layer_ms(r, c) for r, c in shapes]
+        issued = [est[i] for i, _ in plan]
+        assert issued == sorted(issued, reverse=True)
+        load = [0.0] * n_streams
+        for i, k in plan:
+            load[k] += est[i]
+        assert max(load) <= sum(est) / n_streams + max(est) + 1e-9
+    assert ptq.plan_layer_set(shapes[:5], 2, longest_first=False) == [(0, 0), (1, 1), (2, 0), (3, 1), (4, 0)]
+    # wider and taller layers are estimated longer
+    assert ptq.estimate_layer_ms(512, 4608) > ptq.estimate_layer_ms(256, 2304) > ptq.estimate_layer_ms(64, 64)
+    assert ptq.estimate_layer_ms(4096, 4096) > ptq.estimate_layer_ms(512, 4096)
