@@ -20,7 +20,8 @@
  *   - Host-side state (SM count, kernel attributes) is kept per device and looked up with the caller's current
  *     device, so one process may drive several devices; calls may come from several host threads as long as calls
  *     that share a stream, a workspace or output buffers are ordered by the caller.
- *   - Size limits: ptq_quantize_layer takes rows <= 65535 and cols <= 65535 (PTQ_ERR_UNSUPPORTED beyond).
+ *   - Size limits: ptq_quantize_layer (and its dynamic variant) takes rows <= 65535 and cols <= 65535, ptq_prepare_hinv
+ *     cols <= 65535 (PTQ_ERR_UNSUPPORTED beyond).
  *   - No exceptions, no exit(), no stdout, no device trap, no unbounded device-side wait.
  */
 #ifndef PTQ_H_

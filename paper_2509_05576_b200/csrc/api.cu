@@ -323,6 +323,7 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!H || !Hinv || !Hinv_diag || !lambda_out || cols < 1 || !(damp >= 0.0)) return PTQ_ERR_INVALID_ARG;
     if (damp_mode != PTQ_DAMP_REL_MEAN_DIAG && damp_mode != PTQ_DAMP_ABS) return PTQ_ERR_INVALID_ARG;
+    if (cols > kMaxGridY) return PTQ_ERR_UNSUPPORTED;                          // rows index the grid's y dimension
     if (!aligned16(H) || !aligned16(Hinv) || !aligned16(ws)) return PTQ_ERR_ALIGNMENT;
     if (!ws || ws_bytes < ptq_workspace_bytes(PTQ_CALL_PREPARE_HINV, 0, cols, 0)) return PTQ_ERR_WORKSPACE;
     const int n = cols;
@@ -333,7 +334,7 @@ int ptq_prepare_hinv(const double* H, int cols, int damp_mode, double damp, doub
     double* Dbuf = cv.take<double>(chol_scratch_doubles(n));
     void* pws = chol_panel_workspace_bytes(n) ? static_cast<void*>(cv.take<char>(chol_panel_workspace_bytes(n))) : nullptr;
     { Launch l(K_LAMBDA, stream); lambda_kernel<<<1, 256, 0, stream>>>(H, n, damp_mode, damp, lambda_out, status); }
-    { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<148 * 8, 256, 0, stream>>>(H, R, n, lambda_out); }
+    { Launch l(K_DAMP_COPY, stream); damp_copy_kernel<<<dim3(grid_x_for(n, 256), n), 256, 0, stream>>>(H, R, n, lambda_out); }
     // W = U^-T comes out of the factorisation sweep itself (V must start as zero)
     if (cudaMemsetAsync(V, 0, (size_t)n * n * sizeof(double), stream) != cudaSuccess) return PTQ_ERR_CUDA;
     int st = cholesky_upper_auto(R, n, V, Dbuf, bar, pws, status, stream);

@@ -30,16 +30,15 @@ __global__ void __launch_bounds__(256) lambda_kernel(const double* __restrict__ 
     if (threadIdx.x == 0) *lambda_out = mode == PTQ_DAMP_REL_MEAN_DIAG ? damp * (red[0] / (double)n) : damp;
 }
 
-// A = H + lambda I
+// A = H + lambda I, from each row's 64-column diagonal tile on (the factorisation reads the upper triangle only, whole
+// tiles on the diagonal); one grid row per matrix row.
 __global__ void damp_copy_kernel(const double* __restrict__ H, double* __restrict__ A, int n,
                                  const double* __restrict__ lambda) {
-    const int64_t total = (int64_t)n * n;
+    const int i = blockIdx.y;
     const double lam = *lambda;
-    for (int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; idx < total;
-         idx += (int64_t)gridDim.x * blockDim.x) {
-        const int i = (int)(idx / n), j = (int)(idx - (int64_t)i * n);
-        A[idx] = H[idx] + (i == j ? lam : 0.0);
-    }
+    const int64_t row = (int64_t)i * n;
+    for (int j = (i & ~(kNB - 1)) + blockIdx.x * blockDim.x + threadIdx.x; j < n; j += gridDim.x * blockDim.x)
+        A[row + j] = H[row + j] + (i == j ? lam : 0.0);
 }
 
 // ------------------------------------------------------------------------------------------------------------
